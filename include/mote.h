@@ -1,0 +1,185 @@
+/*
+ * mote.h -- C ABI of the B200 (sm_100a) forward pass of one Mixture-of-Ternary-Experts FFN layer
+ * (MoTE, arXiv 2506.14435, Section 3.1).
+ *
+ *     out = [residual +] FFN(x) + sum_{j<k} w_j * FFN^T_{e_j}(x)            (Eq. 2, Eq. 4)
+ *
+ * FFN is the bf16 shared SwiGLU expert; FFN^T_e are routed GLU experts whose weights are ternary
+ * {-1,0,1} with one absmean scale per matrix (Eq. 7, 9) and whose inputs are per-token absmax int8
+ * (Eq. 8).  Ternary weights are stored as INT2 (Section 3.1, last paragraph).
+ *
+ * General rules for every entry point
+ *   - Pointers are DEVICE pointers unless an argument name ends in `_host`.  The caller owns all
+ *     memory; the library never allocates or frees device memory and never synchronises
+ *     (exception: mote_moe_forward_host, documented below).
+ *   - All work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = default stream).
+ *   - Every function returns a mote_status_t.  Argument errors are detected on the host BEFORE
+ *     anything is launched.  A failed launch maps to MOTE_ERR_CUDA.  No exceptions, no exit().
+ *   - bf16 tensors are raw 16-bit patterns.  Matrices are row-major; a weight matrix is W[m, n]
+ *     with n the reduction ("in") dimension, y = W x.
+ *   - Non-finite inputs give undefined results.
+ */
+#ifndef MOTE_H_
+#define MOTE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  MOTE_OK = 0,
+  MOTE_ERR_NULL = 1,           /* a required pointer is NULL                                   */
+  MOTE_ERR_SHAPE = 2,          /* unsupported size (see each call)                              */
+  MOTE_ERR_ALIGN = 3,          /* a pointer or row stride is not 16-byte aligned                */
+  MOTE_ERR_WORKSPACE = 4,      /* workspace missing or too small                                */
+  MOTE_ERR_DTYPE = 5,          /* unknown dtype code                                            */
+  MOTE_ERR_CUDA = 6,           /* a CUDA call or launch failed                                  */
+  MOTE_ERR_DEVICE_TIMEOUT = 7  /* a bounded device-side wait expired (see mote_device_status)   */
+} mote_status_t;
+
+enum { MOTE_DTYPE_F32 = 0, MOTE_DTYPE_BF16 = 1 };
+enum { MOTE_MAX_EXPERTS = 64, MOTE_MAX_TOPK = 8 };
+
+/* Which implementation the expert GEMMs use.  AUTO picks per shape; the others force one path
+ * (used by the tests to check every path against the oracle). */
+enum { MOTE_PATH_AUTO = 0, MOTE_PATH_SIMT = 1, MOTE_PATH_TENSOR = 2, MOTE_PATH_STREAM = 3 };
+
+const char* mote_status_string(mote_status_t st);
+
+/* ------------------------------------------------------------------------------------------------
+ * mote_ternarize_pack -- absmean ternary weight quantizer and INT2 packing (Eq. 7, 9, 10; storage
+ * per Section 3.1).  Offline step, once per matrix.
+ *
+ *   alpha  = max( fl32( (exact sum of |w|) / (m*n) ), 1e-5 )   the sum is exact (integer
+ *            accumulation of fp32 significands), so alpha does not depend on thread order
+ *   code   = clamp( rint( w / alpha ), -1, 1 )                 true fp32 division, ties to even
+ *   packed : m * n/4 bytes; stored value u = code + 1; 4 consecutive elements of a row per byte,
+ *            element j in bits [2*(j%4), 2*(j%4)+1]
+ *
+ *   W        in   [m, n] row-major, dtype w_dtype (MOTE_DTYPE_F32 or MOTE_DTYPE_BF16), 16-B aligned
+ *   packed   out  [m, n/4] uint8, 16-B aligned
+ *   alpha    out  1 float
+ *   ws       scratch of at least mote_ternarize_workspace_bytes() bytes, 16-B aligned
+ * Errors: NULL -> ERR_NULL; m<=0, n<=0, n%16 != 0, m*n >= 2^38 -> ERR_SHAPE; bad dtype -> ERR_DTYPE.
+ */
+size_t mote_ternarize_workspace_bytes(void);
+mote_status_t mote_ternarize_pack(const void* W, int w_dtype, int64_t m, int64_t n,
+                                  uint8_t* packed, float* alpha,
+                                  void* ws, size_t ws_bytes, void* stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * mote_quant_act -- per-token absmax int8 activation quantizer (Eq. 8, 9, 10).
+ *
+ *   beta_t = max( max_j |x[t,j]|, 1e-5 );   q[t,j] = clamp( rint( (127 * x[t,j]) / beta_t ), -128, 127 )
+ *   (127*x exact in fp32, true fp32 division, ties to even);  rowsum[t] = sum_j q[t,j]
+ *
+ *   x_bf16  in   [T, d] bf16, row stride ldx elements (ldx >= d, ldx % 8 == 0), 16-B aligned
+ *   q       out  [T, d] int8 contiguous, 16-B aligned
+ *   beta    out  [T] float
+ *   rowsum  out  [T] int32, may be NULL
+ * T = 0 is a no-op.  Errors: d<=0, d%16 != 0, d > 32768, T<0 -> ERR_SHAPE.
+ */
+mote_status_t mote_quant_act(const void* x_bf16, int64_t T, int64_t d, int64_t ldx,
+                             int8_t* q, float* beta, int32_t* rowsum, void* stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * mote_route_topk -- router of Eq. 3 with top-k selection (no capacity limit, no token dropping).
+ *
+ *   logits[t,e] = sum_j x[t,j] * Wr[e,j] (+ bias[e])        fp32 accumulation
+ *   selection   : the k largest logits, ties to the lower expert index, listed in descending order
+ *   norm_topk=1 : w = softmax over the k selected logits (sums to 1)
+ *   norm_topk=0 : w = P(x)_e of Eq. 3 (softmax over all E experts)
+ *
+ *   x_bf16 [T,d] bf16 contiguous (16-B aligned), Wr [E,d] fp32, bias [E] fp32 or NULL,
+ *   topk_idx [T,k] int32, topk_w [T,k] float, logits [T,E] float or NULL.
+ * Errors: E<1, E>MOTE_MAX_EXPERTS, k<1, k>E, k>MOTE_MAX_TOPK, d%8 != 0 -> ERR_SHAPE.
+ */
+mote_status_t mote_route_topk(const void* x_bf16, int64_t T, int64_t d,
+                              const float* Wr, const float* bias, int E, int k, int norm_topk,
+                              int32_t* topk_idx, float* topk_w, float* logits, void* stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * Layer description (Eq. 2-6).  All device pointers, immutable while calls are in flight.
+ */
+typedef struct {
+  int32_t d, f, E, k, norm_topk;
+  int32_t path;                    /* MOTE_PATH_*                                               */
+  const float* Wr;                 /* [E, d] router projection                                  */
+  const float* router_bias;        /* [E] or NULL                                               */
+  const uint8_t* gate_packed;      /* [E][f, d/4]  packed W_gate of every routed expert          */
+  const uint8_t* up_packed;        /* [E][f, d/4]                                               */
+  const uint8_t* down_packed;      /* [E][d, f/4]                                               */
+  const float* alpha_gate;         /* [E]                                                       */
+  const float* alpha_up;           /* [E]                                                       */
+  const float* alpha_down;         /* [E]                                                       */
+  const void* sh_gate;             /* bf16 [f, d]  shared expert                                */
+  const void* sh_up;               /* bf16 [f, d]                                               */
+  const void* sh_down;             /* bf16 [d, f]                                               */
+} mote_layer_t;
+
+/* Optional copies of intermediates (for parity checks).  Every member may be NULL; a non-NULL
+ * member is filled.  Row-indexed taps are in expert-sorted order: row r = perm[t*k + j]. */
+typedef struct {
+  int32_t* topk_idx;   /* [T, k]                                                                */
+  float* topk_w;       /* [T, k]                                                                */
+  int32_t* offsets;    /* [E+1]   first sorted row of each expert                               */
+  int32_t* perm;       /* [T*k]   pair (t*k+j) -> sorted row                                    */
+  int8_t* qx;          /* [T, d]  Q_a(x) codes, token order                                     */
+  float* beta_x;       /* [T]                                                                   */
+  int32_t* acc_gate;   /* [P, f]  integer accumulators codes_gate . qx                          */
+  int32_t* acc_up;     /* [P, f]                                                                */
+  void* h_bf16;        /* [P, f]  u * SiLU(g), bf16                                             */
+  int8_t* qh;          /* [P, f]  Q_a(h) codes                                                  */
+  float* beta_h;       /* [P]                                                                   */
+  int32_t* acc_down;   /* [P, d]                                                                */
+  float* y;            /* [P, d]  routed expert outputs before gating                           */
+  float* shared_out;   /* [T, d]  FFN(x) of the shared expert                                   */
+} mote_taps_t;
+
+/* Bytes of scratch mote_moe_forward needs for up to T_max tokens (0 if the shape is invalid). */
+size_t mote_workspace_bytes(int d, int f, int E, int k, int64_t T_max);
+
+/* ------------------------------------------------------------------------------------------------
+ * mote_moe_forward -- the whole layer (Eq. 2-8): route, dispatch, Q_a(x), gate/up ternary GEMM
+ * with fused dequantisation and SwiGLU, Q_a(h), down ternary GEMM, shared bf16 FFN, gate-weighted
+ * combine with the shared output and the optional residual.
+ *
+ *   x_bf16         in   [T, d] bf16 contiguous, 16-B aligned
+ *   residual_bf16  in   [T, d] bf16 or NULL; may alias out_bf16
+ *   out_bf16       out  [T, d] bf16; must not alias x_bf16
+ *   taps           NULL or a struct of optional outputs
+ *   ws, ws_bytes   scratch, >= mote_workspace_bytes(d,f,E,k,T), 256-B aligned
+ * Pinned arithmetic: per sorted row, g = fl32(acc_g) * (alpha_g * (beta/127)), u likewise,
+ * h = bf16_rn(u * silu(g)) with silu evaluated by a fixed fp32 sequence, so that the integer
+ * stages that follow are reproducible bit for bit.
+ * T = 0 is a no-op.  Errors: d%16, f%16 != 0, E/k out of range -> ERR_SHAPE; ERR_WORKSPACE;
+ * ERR_ALIGN; path = MOTE_PATH_TENSOR with d%128 or f%128 != 0 -> ERR_SHAPE.
+ */
+mote_status_t mote_moe_forward(const mote_layer_t* L, const void* x_bf16,
+                               const void* residual_bf16, int64_t T, void* out_bf16,
+                               const mote_taps_t* taps, void* ws, size_t ws_bytes, void* stream);
+
+/* Same layer with HOST input and output: copies x_host (and residual_host if non-NULL) to the
+ * device, runs mote_moe_forward, copies the result to out_host and waits for the stream.  Host
+ * buffers should be page-locked for the copies to be asynchronous.  Needs
+ * mote_workspace_bytes(...) + mote_host_staging_bytes(d, T) bytes of device scratch. */
+size_t mote_host_staging_bytes(int d, int64_t T_max);
+mote_status_t mote_moe_forward_host(const mote_layer_t* L, const void* x_host,
+                                    const void* residual_host, int64_t T, void* out_host,
+                                    void* ws, size_t ws_bytes, void* stream);
+
+/* Reads (and clears) the device status word kept at the start of a workspace after the stream has
+ * been synchronised by the caller: MOTE_OK, or MOTE_ERR_DEVICE_TIMEOUT if a kernel gave up a
+ * bounded wait.  Synchronises the stream itself. */
+mote_status_t mote_device_status(void* ws, void* stream);
+
+/* Number of kernels the last mote_moe_forward call on this thread enqueued. */
+int mote_last_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MOTE_H_ */

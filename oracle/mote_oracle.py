@@ -294,7 +294,8 @@ def shared_ffn(x_bf16, Wg_bf16, Wu_bf16, Wd_bf16) -> np.ndarray:
 # --------------------------------------------------------------------------------------------
 
 
-def moe_forward(layer: dict, x_bf16: np.ndarray, residual_bf16=None, token_subset=None):
+def moe_forward(layer: dict, x_bf16: np.ndarray, residual_bf16=None, token_subset=None,
+                near_tie_choice=None):
     """out = [residual +] FFN(x) + sum_j w_j * FFN^T_{e_j}(x)   (Eq. 2 and Eq. 4).
 
     layer: dict with d, f, E, k, norm_topk, Wr[E,d] f32, router_bias[E] f32 or None,
@@ -305,10 +306,22 @@ def moe_forward(layer: dict, x_bf16: np.ndarray, residual_bf16=None, token_subse
       dispatch are still computed for every token.  Row-indexed results are then in the order
       of the subset's pairs sorted by (expert, token, slot); `rows` gives their rows in the
       full dispatch.
+    near_tie_choice: optional int32[T, k].  For the tokens the router flags as near ties (k-th
+      and (k+1)-th logit closer than 1e-5, where an fp32 router may legitimately pick the other
+      expert) the selection is taken from this array instead, and the gate weights are
+      recomputed from the oracle's own logits; every other token keeps the oracle's selection.
     Returns a dict of every intermediate named after the stages above."""
     E, k = layer["E"], layer["k"]
     T, d = x_bf16.shape
     r = router(x_bf16, layer["Wr"], layer.get("router_bias"), k, layer["norm_topk"])
+    if near_tie_choice is not None and r["near_tie"].any():
+        for t in np.nonzero(r["near_tie"])[0]:
+            sel_idx = np.asarray(near_tie_choice[t], dtype=np.int32)
+            lg = r["logits"][t]
+            ex = np.exp(lg[sel_idx] - lg.max())
+            denom = ex.sum() if layer["norm_topk"] else np.exp(lg - lg.max()).sum()
+            r["idx"][t] = sel_idx
+            r["w"][t] = ex / denom
     offsets, perm, inv = dispatch(r["idx"], E)
     qx, beta_x, rowsum_x = quant_act(x_bf16)
 

@@ -1,0 +1,227 @@
+"""ctypes binding of libmote.so.  Argument marshalling only: every step of the layer runs in the
+library's kernels.  torch is used for device memory and streams."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libmote.so")
+if not os.path.exists(_LIB_PATH):
+    raise ImportError(f"{_LIB_PATH} is missing: build it with `python -m paper_2506_14435_b200.build`; "
+                      "there is no fallback path")
+lib = C.CDLL(_LIB_PATH)
+
+PATH_AUTO, PATH_SIMT, PATH_TENSOR, PATH_STREAM = 0, 1, 2, 3
+DTYPE_F32, DTYPE_BF16 = 0, 1
+
+
+class mote_layer_t(C.Structure):
+    _fields_ = [("d", C.c_int32), ("f", C.c_int32), ("E", C.c_int32), ("k", C.c_int32),
+                ("norm_topk", C.c_int32), ("path", C.c_int32),
+                ("Wr", C.c_void_p), ("router_bias", C.c_void_p),
+                ("gate_packed", C.c_void_p), ("up_packed", C.c_void_p), ("down_packed", C.c_void_p),
+                ("alpha_gate", C.c_void_p), ("alpha_up", C.c_void_p), ("alpha_down", C.c_void_p),
+                ("sh_gate", C.c_void_p), ("sh_up", C.c_void_p), ("sh_down", C.c_void_p)]
+
+
+TAP_FIELDS = ["topk_idx", "topk_w", "offsets", "perm", "qx", "beta_x", "acc_gate", "acc_up", "h_bf16",
+              "qh", "beta_h", "acc_down", "y", "shared_out"]
+
+
+class mote_taps_t(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in TAP_FIELDS]
+
+
+lib.mote_status_string.restype = C.c_char_p
+lib.mote_status_string.argtypes = [C.c_int]
+lib.mote_ternarize_workspace_bytes.restype = C.c_size_t
+lib.mote_ternarize_workspace_bytes.argtypes = []
+lib.mote_ternarize_pack.restype = C.c_int
+lib.mote_ternarize_pack.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p,
+                                    C.c_void_p, C.c_size_t, C.c_void_p]
+lib.mote_quant_act.restype = C.c_int
+lib.mote_quant_act.argtypes = [C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p,
+                               C.c_void_p, C.c_void_p]
+lib.mote_route_topk.restype = C.c_int
+lib.mote_route_topk.argtypes = [C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.c_int, C.c_int,
+                                C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+lib.mote_workspace_bytes.restype = C.c_size_t
+lib.mote_workspace_bytes.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, C.c_int64]
+lib.mote_host_staging_bytes.restype = C.c_size_t
+lib.mote_host_staging_bytes.argtypes = [C.c_int, C.c_int64]
+lib.mote_moe_forward.restype = C.c_int
+lib.mote_moe_forward.argtypes = [C.POINTER(mote_layer_t), C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p,
+                                 C.POINTER(mote_taps_t), C.c_void_p, C.c_size_t, C.c_void_p]
+lib.mote_moe_forward_host.restype = C.c_int
+lib.mote_moe_forward_host.argtypes = [C.POINTER(mote_layer_t), C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p,
+                                      C.c_void_p, C.c_size_t, C.c_void_p]
+lib.mote_device_status.restype = C.c_int
+lib.mote_device_status.argtypes = [C.c_void_p, C.c_void_p]
+lib.mote_last_launch_count.restype = C.c_int
+lib.mote_last_launch_count.argtypes = []
+
+
+class MoteError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {lib.mote_status_string(status).decode()} (status {status})")
+
+
+def _check(status: int, where: str):
+    if status != 0:
+        raise MoteError(status, where)
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _need_cuda(*ts):
+    for t in ts:
+        if t is not None and (not t.is_cuda or not t.is_contiguous()):
+            raise ValueError("expected contiguous CUDA tensors")
+
+
+def mote_ternarize_pack(W: torch.Tensor):
+    """Eq. 7, 9: W[m, n] (fp32 or bf16, CUDA) -> (packed uint8[m, n/4], alpha float32[1])."""
+    _need_cuda(W)
+    m, n = W.shape
+    dt = {torch.float32: DTYPE_F32, torch.bfloat16: DTYPE_BF16}[W.dtype]
+    packed = torch.empty((m, max(n // 4, 1)), dtype=torch.uint8, device=W.device)
+    alpha = torch.empty(1, dtype=torch.float32, device=W.device)
+    ws_bytes = lib.mote_ternarize_workspace_bytes()
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=W.device)
+    _check(lib.mote_ternarize_pack(_ptr(W), dt, m, n, _ptr(packed), _ptr(alpha), _ptr(ws), ws_bytes, _stream()),
+           "mote_ternarize_pack")
+    return packed, alpha
+
+
+def mote_quant_act(x: torch.Tensor, want_rowsum: bool = True):
+    """Eq. 8: x[T, d] bf16 (CUDA; rows may be strided) -> (q int8[T,d], beta f32[T], rowsum i32[T])."""
+    if not x.is_cuda or x.dtype != torch.bfloat16 or x.stride(1) != 1:
+        raise ValueError("expected a CUDA bf16 matrix with unit inner stride")
+    T, d = x.shape
+    q = torch.empty((T, d), dtype=torch.int8, device=x.device)
+    beta = torch.empty(T, dtype=torch.float32, device=x.device)
+    rowsum = torch.empty(T, dtype=torch.int32, device=x.device) if want_rowsum else None
+    _check(lib.mote_quant_act(_ptr(x), T, d, x.stride(0) if T > 1 else d, _ptr(q), _ptr(beta), _ptr(rowsum),
+                              _stream()), "mote_quant_act")
+    return q, beta, rowsum
+
+
+def mote_route_topk(x, Wr, bias, k: int, norm_topk: int = 1, want_logits: bool = False):
+    """Eq. 3: returns (topk_idx int32[T,k], topk_w f32[T,k], logits f32[T,E] or None)."""
+    _need_cuda(x, Wr, bias)
+    T, d = x.shape
+    E = Wr.shape[0]
+    idx = torch.empty((T, k), dtype=torch.int32, device=x.device)
+    w = torch.empty((T, k), dtype=torch.float32, device=x.device)
+    logits = torch.empty((T, E), dtype=torch.float32, device=x.device) if want_logits else None
+    _check(lib.mote_route_topk(_ptr(x), T, d, _ptr(Wr), _ptr(bias), E, k, norm_topk, _ptr(idx), _ptr(w),
+                               _ptr(logits), _stream()), "mote_route_topk")
+    return idx, w, logits
+
+
+class MoteLayer:
+    """Device-resident weights of one MoTE layer plus its mote_layer_t."""
+
+    def __init__(self, d, f, E, k, norm_topk, Wr, router_bias, gate_packed, up_packed, down_packed,
+                 alpha_gate, alpha_up, alpha_down, sh_gate, sh_up, sh_down, path=PATH_AUTO):
+        self.d, self.f, self.E, self.k, self.norm_topk, self.path = d, f, E, k, norm_topk, path
+        self.tensors = dict(Wr=Wr, router_bias=router_bias, gate_packed=gate_packed, up_packed=up_packed,
+                            down_packed=down_packed, alpha_gate=alpha_gate, alpha_up=alpha_up,
+                            alpha_down=alpha_down, sh_gate=sh_gate, sh_up=sh_up, sh_down=sh_down)
+        _need_cuda(*self.tensors.values())
+        self._ws = None
+
+    @classmethod
+    def from_master(cls, master: dict, device="cuda", path=PATH_AUTO):
+        """Offline step: upload fp32 master weights (numpy, see workloads.synth.master_layer) and
+        ternarize every routed matrix on the device with mote_ternarize_pack."""
+        d, f, E = master["d"], master["f"], master["E"]
+        dev = torch.device(device)
+        packed = {}
+        alphas = {}
+        for name, shape in (("gate", (f, d)), ("up", (f, d)), ("down", (d, f))):
+            buf = torch.empty((E, shape[0], shape[1] // 4), dtype=torch.uint8, device=dev)
+            al = torch.empty(E, dtype=torch.float32, device=dev)
+            for e in range(E):
+                W = torch.from_numpy(master["W_" + name][e]).to(dev)
+                p, a = mote_ternarize_pack(W)
+                buf[e].copy_(p)
+                al[e:e + 1].copy_(a)
+            packed[name], alphas[name] = buf, al
+
+        def bf16(bits):
+            return torch.from_numpy(bits.view("int16")).view(torch.bfloat16).to(dev)
+
+        bias = master.get("router_bias")
+        return cls(d, f, E, master["k"], master["norm_topk"], torch.from_numpy(master["Wr"]).to(dev),
+                   None if bias is None else torch.from_numpy(bias).to(dev),
+                   packed["gate"], packed["up"], packed["down"], alphas["gate"], alphas["up"], alphas["down"],
+                   bf16(master["sh_gate"]), bf16(master["sh_up"]), bf16(master["sh_down"]), path=path)
+
+    def struct(self) -> mote_layer_t:
+        t = self.tensors
+        s = mote_layer_t(self.d, self.f, self.E, self.k, self.norm_topk, self.path)
+        for name in ("Wr", "router_bias", "gate_packed", "up_packed", "down_packed", "alpha_gate", "alpha_up",
+                     "alpha_down", "sh_gate", "sh_up", "sh_down"):
+            setattr(s, name, None if t[name] is None else t[name].data_ptr())
+        return s
+
+    def workspace(self, T: int, host_staging: bool = False) -> torch.Tensor:
+        need = lib.mote_workspace_bytes(self.d, self.f, self.E, self.k, T)
+        if need == 0:
+            raise MoteError(2, "mote_workspace_bytes")
+        if host_staging:
+            need += lib.mote_host_staging_bytes(self.d, T)
+        if self._ws is None or self._ws.numel() < need:
+            self._ws = torch.empty(need, dtype=torch.uint8, device=self.tensors["Wr"].device)
+        return self._ws
+
+    def alloc_taps(self, T: int, names=TAP_FIELDS):
+        dev = self.tensors["Wr"].device
+        P, d, f, E, k = T * self.k, self.d, self.f, self.E, self.k
+        spec = dict(topk_idx=((T, k), torch.int32), topk_w=((T, k), torch.float32),
+                    offsets=((E + 1,), torch.int32), perm=((P,), torch.int32), qx=((T, d), torch.int8),
+                    beta_x=((T,), torch.float32), acc_gate=((P, f), torch.int32), acc_up=((P, f), torch.int32),
+                    h_bf16=((P, f), torch.bfloat16), qh=((P, f), torch.int8), beta_h=((P,), torch.float32),
+                    acc_down=((P, d), torch.int32), y=((P, d), torch.float32),
+                    shared_out=((T, d), torch.float32))
+        return {n: torch.zeros(spec[n][0], dtype=spec[n][1], device=dev) for n in names}
+
+
+def mote_moe_forward(layer: MoteLayer, x: torch.Tensor, residual=None, out=None, taps: dict | None = None):
+    """Eq. 2-8 for x[T, d] bf16 (CUDA).  Returns out[T, d] bf16; fills the tensors in `taps`."""
+    _need_cuda(x, residual, out)
+    T = x.shape[0]
+    if out is None:
+        out = torch.empty_like(x)
+    ws = layer.workspace(T)
+    s = layer.struct()
+    tp = None
+    if taps is not None:
+        tp = mote_taps_t()
+        for n, t in taps.items():
+            setattr(tp, n, t.data_ptr())
+        tp = C.byref(tp)
+    _check(lib.mote_moe_forward(C.byref(s), _ptr(x), _ptr(residual), T, _ptr(out), tp, _ptr(ws), ws.numel(),
+                                _stream()), "mote_moe_forward")
+    return out
+
+
+def mote_moe_forward_host(layer: MoteLayer, x_host: torch.Tensor, out_host: torch.Tensor, residual_host=None):
+    """Same layer with (pinned) host tensors in and out; synchronises the stream."""
+    T = x_host.shape[0]
+    ws = layer.workspace(T, host_staging=True)
+    s = layer.struct()
+    _check(lib.mote_moe_forward_host(C.byref(s), _ptr(x_host), _ptr(residual_host), T, _ptr(out_host), _ptr(ws),
+                                     ws.numel(), _stream()), "mote_moe_forward_host")
+    return out_host

@@ -1,0 +1,257 @@
+// Host side of mote_moe_forward: argument checks, workspace plan, launch sequence (Eq. 2-8).
+//
+//   S1 route -> S2 dispatch -> S3 Q_a(x) scattered to expert-sorted rows -> S4 gate/up ternary
+//   GEMM (+dequant, SwiGLU) -> S5 Q_a(h) -> S6 down ternary GEMM -> S7 shared bf16 FFN ->
+//   S8 combine.  Everything is enqueued on the caller's stream; nothing synchronises.
+#include <algorithm>
+
+#include "mote_common.cuh"
+#include "mote_internal.h"
+
+namespace mote {
+
+thread_local int g_launch_count = 0;
+
+struct Plan {
+  size_t status, topk_idx, topk_w, offsets, perm, inv;
+  size_t qx, beta_x, rowsum_x, h, qh, beta_h, rowsum_h, y, hs, s;
+  size_t total;
+};
+
+static Plan make_plan(int d, int f, int E, int k, int64_t T) {
+  Plan p{};
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off += round_up(std::max<size_t>(bytes, 1), 256); return o; };
+  const size_t P = size_t(T) * k;
+  p.status = take(256);
+  p.topk_idx = take(P * 4);
+  p.topk_w = take(P * 4);
+  p.offsets = take(size_t(E + 1) * 4);
+  p.perm = take(P * 4);
+  p.inv = take(P * 4);
+  p.qx = take(P * size_t(d));
+  p.beta_x = take(P * 4);
+  p.rowsum_x = take(P * 4);
+  p.h = take(P * size_t(f) * 2);
+  p.qh = take(P * size_t(f));
+  p.beta_h = take(P * 4);
+  p.rowsum_h = take(P * 4);
+  p.y = take(P * size_t(d) * 4);
+  p.hs = take(size_t(T) * f * 2);
+  p.s = take(size_t(T) * d * 4);
+  p.total = off;
+  return p;
+}
+
+static bool shape_ok(int d, int f, int E, int k) {
+  return d > 0 && f > 0 && d % 16 == 0 && f % 16 == 0 && d <= 32768 && f <= 32768 && E >= 1 &&
+         E <= MOTE_MAX_EXPERTS && k >= 1 && k <= E && k <= MOTE_MAX_TOPK;
+}
+
+// Copies int8 rows, undoing the k-interleaved storage of each 16-code unit when asked, with an
+// optional row map (dst row r <- src row map[r * map_stride]).
+__global__ void copy_q_rows_kernel(const int8_t* __restrict__ src, int8_t* __restrict__ dst, int64_t rows,
+                                   int n_units, const int32_t* __restrict__ map, int map_stride, int deinterleave) {
+  const int64_t total = rows * n_units;
+  const int64_t stride = int64_t(gridDim.x) * blockDim.x;
+  for (int64_t i = int64_t(blockIdx.x) * blockDim.x + threadIdx.x; i < total; i += stride) {
+    const int64_t r = i / n_units;
+    const int u = (int)(i - r * n_units);
+    const int64_t sr = map ? int64_t(map[r * map_stride]) : r;
+    uint4 v = reinterpret_cast<const uint4*>(src)[sr * n_units + u];
+    if (deinterleave) {
+      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+      uint32_t o[4];
+#pragma unroll
+      for (int b = 0; b < 4; ++b)
+        o[b] = ((w[0] >> (8 * b)) & 0xFFu) | (((w[1] >> (8 * b)) & 0xFFu) << 8) |
+               (((w[2] >> (8 * b)) & 0xFFu) << 16) | (((w[3] >> (8 * b)) & 0xFFu) << 24);
+      v = make_uint4(o[0], o[1], o[2], o[3]);
+    }
+    reinterpret_cast<uint4*>(dst)[r * n_units + u] = v;
+  }
+}
+
+__global__ void gather_f32_kernel(const float* __restrict__ src, float* __restrict__ dst, int64_t n,
+                                  const int32_t* __restrict__ map, int map_stride) {
+  const int64_t i = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (i < n) dst[i] = src[map[i * map_stride]];
+}
+
+}  // namespace mote
+
+using namespace mote;
+
+extern "C" const char* mote_status_string(mote_status_t st) {
+  switch (st) {
+    case MOTE_OK: return "ok";
+    case MOTE_ERR_NULL: return "null pointer";
+    case MOTE_ERR_SHAPE: return "unsupported shape";
+    case MOTE_ERR_ALIGN: return "misaligned pointer or stride";
+    case MOTE_ERR_WORKSPACE: return "workspace missing or too small";
+    case MOTE_ERR_DTYPE: return "unknown dtype";
+    case MOTE_ERR_CUDA: return "CUDA error";
+    case MOTE_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+  }
+  return "unknown status";
+}
+
+extern "C" size_t mote_workspace_bytes(int d, int f, int E, int k, int64_t T_max) {
+  if (!shape_ok(d, f, E, k) || T_max < 0 || T_max > (int64_t(1) << 24)) return 0;
+  return make_plan(d, f, E, k, T_max).total;
+}
+
+extern "C" size_t mote_host_staging_bytes(int d, int64_t T_max) {
+  if (d <= 0 || T_max < 0) return 0;
+  return 3 * round_up(size_t(T_max) * d * 2, 256);
+}
+
+extern "C" int mote_last_launch_count(void) { return g_launch_count; }
+
+extern "C" mote_status_t mote_device_status(void* ws, void* stream_) {
+  if (!ws) return MOTE_ERR_NULL;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  uint32_t word = 0;
+  MOTE_CUDA_OK(cudaMemcpyAsync(&word, ws, sizeof(word), cudaMemcpyDeviceToHost, stream));
+  MOTE_CUDA_OK(cudaStreamSynchronize(stream));
+  if (word != 0) {
+    MOTE_CUDA_OK(cudaMemsetAsync(ws, 0, sizeof(word), stream));
+    return MOTE_ERR_DEVICE_TIMEOUT;
+  }
+  return MOTE_OK;
+}
+
+extern "C" mote_status_t mote_moe_forward(const mote_layer_t* L, const void* x, const void* residual, int64_t T,
+                                          void* out, const mote_taps_t* taps, void* ws, size_t ws_bytes,
+                                          void* stream_) {
+  g_launch_count = 0;
+  if (!L) return MOTE_ERR_NULL;
+  const int d = L->d, f = L->f, E = L->E, k = L->k;
+  if (!shape_ok(d, f, E, k) || T < 0 || T > (int64_t(1) << 24)) return MOTE_ERR_SHAPE;
+  if (L->path < MOTE_PATH_AUTO || L->path > MOTE_PATH_STREAM) return MOTE_ERR_SHAPE;
+  if (T == 0) return MOTE_OK;
+  if (!x || !out || !ws || !L->Wr || !L->gate_packed || !L->up_packed || !L->down_packed || !L->alpha_gate ||
+      !L->alpha_up || !L->alpha_down || !L->sh_gate || !L->sh_up || !L->sh_down)
+    return MOTE_ERR_NULL;
+  if (x == out) return MOTE_ERR_SHAPE;
+  const void* ptrs[] = {x, out, residual, L->Wr, L->gate_packed, L->up_packed, L->down_packed,
+                        L->sh_gate, L->sh_up, L->sh_down};
+  for (const void* p : ptrs)
+    if (p && !aligned16(p)) return MOTE_ERR_ALIGN;
+  if ((reinterpret_cast<uintptr_t>(ws) & 255u) != 0) return MOTE_ERR_ALIGN;
+  const Plan pl = make_plan(d, f, E, k, T);
+  if (ws_bytes < pl.total) return MOTE_ERR_WORKSPACE;
+  const int64_t P = T * k;
+  if ((P + 31) / 32 + E > 65535) return MOTE_ERR_SHAPE;
+
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  char* base = static_cast<char*>(ws);
+  auto* topk_idx = reinterpret_cast<int32_t*>(base + pl.topk_idx);
+  auto* topk_w = reinterpret_cast<float*>(base + pl.topk_w);
+  auto* offsets = reinterpret_cast<int32_t*>(base + pl.offsets);
+  auto* perm = reinterpret_cast<int32_t*>(base + pl.perm);
+  auto* inv = reinterpret_cast<int32_t*>(base + pl.inv);
+  auto* qx = reinterpret_cast<int8_t*>(base + pl.qx);
+  auto* beta_x = reinterpret_cast<float*>(base + pl.beta_x);
+  auto* rowsum_x = reinterpret_cast<int32_t*>(base + pl.rowsum_x);
+  void* h = base + pl.h;
+  auto* qh = reinterpret_cast<int8_t*>(base + pl.qh);
+  auto* beta_h = reinterpret_cast<float*>(base + pl.beta_h);
+  auto* rowsum_h = reinterpret_cast<int32_t*>(base + pl.rowsum_h);
+  auto* y = reinterpret_cast<float*>(base + pl.y);
+  void* hs = base + pl.hs;
+  auto* s = reinterpret_cast<float*>(base + pl.s);
+
+  const int path = (L->path == MOTE_PATH_AUTO) ? MOTE_PATH_SIMT : L->path;
+  if (path != MOTE_PATH_SIMT) return MOTE_ERR_SHAPE;     // other paths are wired in below as they land
+  const int interleave = 0;
+
+  mote_status_t st;
+  // S1 router, S2 dispatch
+  st = launch_route_topk(x, T, d, L->Wr, L->router_bias, E, k, L->norm_topk, topk_idx, topk_w, nullptr, stream);
+  if (st) return st;
+  st = launch_dispatch(topk_idx, P, E, offsets, perm, inv, stream);
+  if (st) return st;
+  // S3 Q_a(x), written once per selected expert into the expert-sorted rows
+  QuantActArgs qa{};
+  qa.x = x; qa.T = T; qa.d = d; qa.ldx = d; qa.q = qx; qa.beta = beta_x; qa.rowsum = rowsum_x;
+  qa.perm = perm; qa.k = k; qa.interleave = interleave;
+  st = launch_quant_act(qa, true, stream);
+  if (st) return st;
+  // S4 gate/up
+  TernaryGemmArgs g1{};
+  g1.qa = qx; g1.beta = beta_x; g1.offsets = offsets; g1.w0 = L->gate_packed; g1.w1 = L->up_packed;
+  g1.alpha0 = L->alpha_gate; g1.alpha1 = L->alpha_up; g1.E = E; g1.N = f; g1.K = d; g1.P = P;
+  g1.h_bf16 = h; g1.acc0_tap = taps ? taps->acc_gate : nullptr; g1.acc1_tap = taps ? taps->acc_up : nullptr;
+  st = launch_ternary_gateup_simt(g1, stream);
+  if (st) return st;
+  // S5 Q_a(h)
+  QuantActArgs qb{};
+  qb.x = h; qb.T = P; qb.d = f; qb.ldx = f; qb.q = qh; qb.beta = beta_h; qb.rowsum = rowsum_h;
+  qb.perm = nullptr; qb.k = 1; qb.interleave = interleave;
+  st = launch_quant_act(qb, false, stream);
+  if (st) return st;
+  // S6 down
+  TernaryGemmArgs g2{};
+  g2.qa = qh; g2.beta = beta_h; g2.offsets = offsets; g2.w0 = L->down_packed; g2.alpha0 = L->alpha_down;
+  g2.E = E; g2.N = d; g2.K = f; g2.P = P; g2.y = y; g2.acc0_tap = taps ? taps->acc_down : nullptr;
+  st = launch_ternary_down_simt(g2, stream);
+  if (st) return st;
+  // S7 shared expert
+  st = launch_shared_gateup_simt(x, L->sh_gate, L->sh_up, T, d, f, hs, stream);
+  if (st) return st;
+  st = launch_shared_down_simt(hs, L->sh_down, T, d, f, s, stream);
+  if (st) return st;
+  // S8 combine
+  st = launch_combine(s, y, topk_w, perm, residual, T, d, k, out, stream);
+  if (st) return st;
+
+  if (taps) {
+    auto d2d = [&](void* dst, const void* src, size_t bytes) -> bool {
+      return !dst || cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToDevice, stream) == cudaSuccess;
+    };
+    bool ok = d2d(taps->topk_idx, topk_idx, P * 4) && d2d(taps->topk_w, topk_w, P * 4) &&
+              d2d(taps->offsets, offsets, size_t(E + 1) * 4) && d2d(taps->perm, perm, P * 4) &&
+              d2d(taps->h_bf16, h, size_t(P) * f * 2) && d2d(taps->beta_h, beta_h, P * 4) &&
+              d2d(taps->y, y, size_t(P) * d * 4) && d2d(taps->shared_out, s, size_t(T) * d * 4);
+    if (!ok) return MOTE_ERR_CUDA;
+    if (taps->qx) {
+      copy_q_rows_kernel<<<148 * 4, 256, 0, stream>>>(qx, taps->qx, T, d / 16, perm, k, interleave);
+      MOTE_LAUNCH_OK();
+    }
+    if (taps->beta_x) {
+      gather_f32_kernel<<<(unsigned)((T + 255) / 256), 256, 0, stream>>>(beta_x, taps->beta_x, T, perm, k);
+      MOTE_LAUNCH_OK();
+    }
+    if (taps->qh) {
+      copy_q_rows_kernel<<<148 * 4, 256, 0, stream>>>(qh, taps->qh, P, f / 16, nullptr, 0, interleave);
+      MOTE_LAUNCH_OK();
+    }
+  }
+  return MOTE_OK;
+}
+
+extern "C" mote_status_t mote_moe_forward_host(const mote_layer_t* L, const void* x_host, const void* residual_host,
+                                               int64_t T, void* out_host, void* ws, size_t ws_bytes, void* stream_) {
+  if (!L) return MOTE_ERR_NULL;
+  if (T < 0) return MOTE_ERR_SHAPE;
+  if (T == 0) return MOTE_OK;
+  if (!x_host || !out_host || !ws) return MOTE_ERR_NULL;
+  const size_t core = mote_workspace_bytes(L->d, L->f, L->E, L->k, T);
+  if (core == 0) return MOTE_ERR_SHAPE;
+  const size_t slab = round_up(size_t(T) * L->d * 2, 256);
+  if (ws_bytes < core + 3 * slab) return MOTE_ERR_WORKSPACE;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  char* stage = static_cast<char*>(ws) + core;
+  void* x_dev = stage;
+  void* res_dev = residual_host ? stage + slab : nullptr;
+  void* out_dev = stage + 2 * slab;
+  const size_t bytes = size_t(T) * L->d * 2;
+  MOTE_CUDA_OK(cudaMemcpyAsync(x_dev, x_host, bytes, cudaMemcpyHostToDevice, stream));
+  if (residual_host) MOTE_CUDA_OK(cudaMemcpyAsync(res_dev, residual_host, bytes, cudaMemcpyHostToDevice, stream));
+  mote_status_t st = mote_moe_forward(L, x_dev, res_dev, T, out_dev, nullptr, ws, core, stream);
+  if (st) return st;
+  MOTE_CUDA_OK(cudaMemcpyAsync(out_host, out_dev, bytes, cudaMemcpyDeviceToHost, stream));
+  MOTE_CUDA_OK(cudaStreamSynchronize(stream));
+  return MOTE_OK;
+}

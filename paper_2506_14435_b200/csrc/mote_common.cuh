@@ -1,0 +1,109 @@
+// Shared host/device helpers of the MoTE sm_100a kernels.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "mote.h"
+
+#define MOTE_CUDA_OK(expr)                                   \
+  do {                                                       \
+    cudaError_t _e = (expr);                                 \
+    if (_e != cudaSuccess) return MOTE_ERR_CUDA;             \
+  } while (0)
+
+#define MOTE_LAUNCH_OK()                                     \
+  do {                                                       \
+    if (cudaGetLastError() != cudaSuccess) return MOTE_ERR_CUDA; \
+  } while (0)
+
+namespace mote {
+
+constexpr float kEpsScale = 1e-5f;  // lower clamp of alpha (Eq. 9) and beta (Eq. 8)
+
+static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+static inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Counts kernel launches of the current forward call (host side, per thread).
+extern thread_local int g_launch_count;
+
+// ---------------------------------------------------------------------------------------------
+// bf16 helpers (bf16 = upper half of an IEEE binary32)
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ float bf16_lo(uint32_t packed2) { return __uint_as_float(packed2 << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t packed2) { return __uint_as_float(packed2 & 0xFFFF0000u); }
+__device__ __forceinline__ float bf16_bits_to_f32(uint16_t b) { return __uint_as_float(uint32_t(b) << 16); }
+
+// round-to-nearest-even fp32 -> bf16 bits (finite inputs)
+__device__ __forceinline__ uint32_t f32_to_bf16_bits(float x) {
+  uint32_t u = __float_as_uint(x);
+  u += 0x7FFFu + ((u >> 16) & 1u);
+  return u >> 16;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Eq. 8: q = clamp(rint((127*x)/beta), -128, 127); 127*x is exact for a bf16 x.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ int quant_one(float x, float beta) {
+  float t = __fmul_rn(127.0f, x);
+  float r = rintf(__fdiv_rn(t, beta));
+  r = fminf(fmaxf(r, -128.0f), 127.0f);
+  return __float2int_rn(r);
+}
+
+// ---------------------------------------------------------------------------------------------
+// SiLU of Eq. 6 as a fixed sequence of single correctly-rounded fp32 operations (no FMA
+// contraction: every multiply and add is an explicit _rn intrinsic).
+//   t = clamp((-g)*log2(e), -125, 125);  n = rint(t);  r = t - n
+//   p = c6;  p = p*r + c_i  (i = 5..0), c_i = fl32(ln2^i / i!)
+//   E = p * 2^n;   silu = g / (1 + E)
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ float exp_neg_pinned(float g) {
+  float t = __fmul_rn(-g, 1.4426950408889634f);
+  t = fminf(fmaxf(t, -125.0f), 125.0f);
+  float n = rintf(t);
+  float r = __fsub_rn(t, n);
+  float p = 1.5403530393381609e-4f;                       // ln2^6/720
+  p = __fadd_rn(__fmul_rn(p, r), 1.3333558146428443e-3f); // ln2^5/120
+  p = __fadd_rn(__fmul_rn(p, r), 9.6181291076284772e-3f); // ln2^4/24
+  p = __fadd_rn(__fmul_rn(p, r), 5.5504108664821580e-2f); // ln2^3/6
+  p = __fadd_rn(__fmul_rn(p, r), 2.4022650695910071e-1f); // ln2^2/2
+  p = __fadd_rn(__fmul_rn(p, r), 6.9314718055994531e-1f); // ln2
+  p = __fadd_rn(__fmul_rn(p, r), 1.0f);
+  float scale = __int_as_float((__float2int_rn(n) + 127) << 23);
+  return __fmul_rn(p, scale);
+}
+
+__device__ __forceinline__ float silu_pinned(float g) {
+  return __fdiv_rn(g, __fadd_rn(1.0f, exp_neg_pinned(g)));
+}
+
+// h = bf16_rn(u * silu(g)),  g = fl32(acc_g) * c_g,  u = fl32(acc_u) * c_u
+__device__ __forceinline__ float glu_h(int acc_g, int acc_u, float c_g, float c_u) {
+  float g = __fmul_rn(__int2float_rn(acc_g), c_g);
+  float u = __fmul_rn(__int2float_rn(acc_u), c_u);
+  return __fmul_rn(u, silu_pinned(g));
+}
+
+// scale of one ternary linear output row: alpha * (beta / 127)
+__device__ __forceinline__ float dequant_scale(float alpha, float beta) {
+  return __fmul_rn(alpha, __fdiv_rn(beta, 127.0f));
+}
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+__device__ __forceinline__ int warp_sum(int v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+}  // namespace mote

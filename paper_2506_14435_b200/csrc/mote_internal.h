@@ -1,0 +1,66 @@
+// Host-side declarations shared by the translation units of libmote (not part of the C ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "mote.h"
+
+namespace mote {
+
+struct QuantActArgs {
+  const void* x;        // bf16 [T, ldx]
+  int64_t T;
+  int d;
+  int64_t ldx;
+  int8_t* q;            // [rows, d]
+  float* beta;          // [rows]
+  int32_t* rowsum;      // [rows] or null
+  const int32_t* perm;  // scatter variant: pair (t*k+j) -> destination row
+  int k;
+  int interleave;       // 1: store each unit of 16 codes k-interleaved
+  int group;            // threads per row (set by the launcher)
+};
+mote_status_t launch_quant_act(const QuantActArgs& a, bool scatter, cudaStream_t stream);
+
+// Router (Eq. 3).  Arguments as mote_route_topk.
+mote_status_t launch_route_topk(const void* x, int64_t T, int d, const float* Wr, const float* bias,
+                                int E, int k, int norm_topk, int32_t* idx, float* w, float* logits,
+                                cudaStream_t stream);
+
+// Stable grouping of the T*k pairs by expert: offsets[E+1], perm[P] (pair -> row), inv[P] (row -> pair).
+mote_status_t launch_dispatch(const int32_t* idx, int64_t P, int E, int32_t* offsets, int32_t* perm,
+                              int32_t* inv, cudaStream_t stream);
+
+// CUDA-core (dp4a) grouped ternary GEMMs.  qa rows are in expert-sorted order, canonical k order.
+struct TernaryGemmArgs {
+  const int8_t* qa;          // [P, K] int8 activations, sorted rows
+  const float* beta;         // [P]
+  const int32_t* offsets;    // [E+1]
+  const uint8_t* w0;         // [E][N, K/4] packed (gate, or down)
+  const uint8_t* w1;         // [E][N, K/4] packed up (gate/up mode) or null
+  const float* alpha0;       // [E]
+  const float* alpha1;       // [E] or null
+  int E, N, K;
+  int64_t P;
+  // outputs
+  void* h_bf16;              // gate/up mode: [P, N] bf16
+  float* y;                  // down mode: [P, N] fp32
+  int32_t* acc0_tap;         // optional [P, N]
+  int32_t* acc1_tap;         // optional [P, N]
+};
+mote_status_t launch_ternary_gateup_simt(const TernaryGemmArgs& a, cudaStream_t stream);
+mote_status_t launch_ternary_down_simt(const TernaryGemmArgs& a, cudaStream_t stream);
+
+// CUDA-core bf16 GEMMs of the shared expert.
+mote_status_t launch_shared_gateup_simt(const void* x, const void* Wg, const void* Wu, int64_t T, int d,
+                                        int f, void* h_bf16, cudaStream_t stream);
+mote_status_t launch_shared_down_simt(const void* h, const void* Wd, int64_t T, int d, int f, float* s,
+                                      cudaStream_t stream);
+
+// out = [residual +] s + sum_j w_j * y[perm[t*k+j]]
+mote_status_t launch_combine(const float* s, const float* y, const float* w, const int32_t* perm,
+                             const void* residual, int64_t T, int d, int k, void* out_bf16,
+                             cudaStream_t stream);
+
+}  // namespace mote

@@ -1,0 +1,162 @@
+// Per-token absmax int8 activation quantizer (Eq. 8-10).
+//
+// One group of G threads (G = 32..256, a power of two) owns one token row and keeps it in
+// registers between the absmax pass and the quantisation pass, so x is read from HBM once.
+// Each thread handles units of 16 consecutive elements: two 128-bit loads in, one 128-bit store
+// out.  HBM-bound: 2 B read + 1 B written per element.
+//
+// The layer-internal variant writes the row to the k expert-sorted positions of its token and
+// can store each unit of 16 codes in the "k-interleaved" order the tensor-core GEMM wants
+// (stored[4*i + b] = q[4*b + i]): the GEMM's 2-bit weight unpacker yields weights in the same
+// order, and an integer dot product does not depend on the order of its terms.
+#include <algorithm>
+
+#include "mote_common.cuh"
+#include "mote_internal.h"
+
+namespace mote {
+
+template <int kUnits, bool kScatter>
+__global__ void __launch_bounds__(256) quant_act_kernel(QuantActArgs a) {
+  __shared__ float s_max[8];
+  __shared__ int s_sum[8];
+  const int G = a.group;                          // threads per row
+  const int rows_per_cta = blockDim.x / G;
+  const int g = threadIdx.x / G;                  // row slot inside the CTA
+  const int tg = threadIdx.x % G;                 // thread inside the group
+  const int64_t row = int64_t(blockIdx.x) * rows_per_cta + g;
+  const bool row_ok = row < a.T;
+  const int n_units = a.d / 16;
+
+  uint4 raw[kUnits][2];
+  float amax = 0.0f;
+  const uint4* src = reinterpret_cast<const uint4*>(
+      reinterpret_cast<const uint16_t*>(a.x) + (row_ok ? row : 0) * a.ldx);
+#pragma unroll
+  for (int u = 0; u < kUnits; ++u) {
+    const int unit = tg + u * G;
+    if (row_ok && unit < n_units) {
+      raw[u][0] = src[unit * 2];
+      raw[u][1] = src[unit * 2 + 1];
+    } else {
+      raw[u][0] = make_uint4(0, 0, 0, 0);
+      raw[u][1] = make_uint4(0, 0, 0, 0);
+    }
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const uint32_t w[4] = {raw[u][h].x, raw[u][h].y, raw[u][h].z, raw[u][h].w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        amax = fmaxf(amax, fabsf(bf16_lo(w[j])));
+        amax = fmaxf(amax, fabsf(bf16_hi(w[j])));
+      }
+    }
+  }
+  // group-wide max
+  amax = warp_max(amax);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (G > 32) {
+    if (lane == 0) s_max[warp] = amax;
+    __syncthreads();
+    const int w0 = (g * G) >> 5, nw = G >> 5;
+    float m = s_max[w0];
+    for (int i = 1; i < nw; ++i) m = fmaxf(m, s_max[w0 + i]);
+    amax = m;
+  }
+  const float beta = fmaxf(amax, kEpsScale);
+
+  int local_sum = 0;
+  uint4 outw[kUnits];
+#pragma unroll
+  for (int u = 0; u < kUnits; ++u) {
+    int q[16];
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const uint32_t w[4] = {raw[u][h].x, raw[u][h].y, raw[u][h].z, raw[u][h].w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        q[h * 8 + 2 * j] = quant_one(bf16_lo(w[j]), beta);
+        q[h * 8 + 2 * j + 1] = quant_one(bf16_hi(w[j]), beta);
+      }
+    }
+    uint32_t o[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      if (a.interleave)
+        o[i] = (q[i] & 0xFF) | ((q[4 + i] & 0xFF) << 8) | ((q[8 + i] & 0xFF) << 16) | ((q[12 + i] & 0xFF) << 24);
+      else
+        o[i] = (q[4 * i] & 0xFF) | ((q[4 * i + 1] & 0xFF) << 8) | ((q[4 * i + 2] & 0xFF) << 16) |
+               ((q[4 * i + 3] & 0xFF) << 24);
+    }
+#pragma unroll
+    for (int j = 0; j < 16; ++j) local_sum += q[j];
+    outw[u] = make_uint4(o[0], o[1], o[2], o[3]);
+  }
+  local_sum = warp_sum(local_sum);
+  if (G > 32) {
+    if (lane == 0) s_sum[warp] = local_sum;
+    __syncthreads();
+    const int w0 = (g * G) >> 5, nw = G >> 5;
+    int s = 0;
+    for (int i = 0; i < nw; ++i) s += s_sum[w0 + i];
+    local_sum = s;
+  }
+  if (!row_ok) return;
+
+  const int n_dst = kScatter ? a.k : 1;
+  for (int j = 0; j < n_dst; ++j) {
+    const int64_t dst = kScatter ? int64_t(a.perm[row * a.k + j]) : row;
+    uint4* out = reinterpret_cast<uint4*>(a.q + dst * int64_t(a.d));
+#pragma unroll
+    for (int u = 0; u < kUnits; ++u) {
+      const int unit = tg + u * G;
+      if (unit < n_units) out[unit] = outw[u];
+    }
+    if (tg == 0) {
+      a.beta[dst] = beta;
+      if (a.rowsum) a.rowsum[dst] = local_sum;
+    }
+  }
+}
+
+mote_status_t launch_quant_act(const QuantActArgs& a, bool scatter, cudaStream_t stream) {
+  if (a.T == 0) return MOTE_OK;
+  const int n_units = a.d / 16;
+  // smallest power-of-two group with at most 4 units per thread (8 for the widest rows)
+  int G = 32;
+  while (G < 256 && n_units > G * 4) G <<= 1;
+  const int upt = (n_units + G - 1) / G;
+  QuantActArgs args = a;
+  args.group = G;
+  const int threads = 256;
+  const int rows_per_cta = threads / G;
+  const unsigned blocks = (unsigned)((a.T + rows_per_cta - 1) / rows_per_cta);
+#define MOTE_QA_LAUNCH(U)                                                          \
+  do {                                                                             \
+    if (scatter) quant_act_kernel<U, true><<<blocks, threads, 0, stream>>>(args);  \
+    else quant_act_kernel<U, false><<<blocks, threads, 0, stream>>>(args);         \
+  } while (0)
+  if (upt <= 1) MOTE_QA_LAUNCH(1);
+  else if (upt <= 2) MOTE_QA_LAUNCH(2);
+  else if (upt <= 4) MOTE_QA_LAUNCH(4);
+  else MOTE_QA_LAUNCH(8);
+#undef MOTE_QA_LAUNCH
+  ++g_launch_count;
+  MOTE_LAUNCH_OK();
+  return MOTE_OK;
+}
+
+}  // namespace mote
+
+extern "C" mote_status_t mote_quant_act(const void* x_bf16, int64_t T, int64_t d, int64_t ldx,
+                                        int8_t* q, float* beta, int32_t* rowsum, void* stream) {
+  using namespace mote;
+  if (T < 0 || d <= 0 || (d % 16) != 0 || d > 32768 || ldx < d || (ldx % 8) != 0) return MOTE_ERR_SHAPE;
+  if (T == 0) return MOTE_OK;
+  if (!x_bf16 || !q || !beta) return MOTE_ERR_NULL;
+  if (!aligned16(x_bf16) || !aligned16(q)) return MOTE_ERR_ALIGN;
+  QuantActArgs a{};
+  a.x = x_bf16; a.T = T; a.d = (int)d; a.ldx = ldx; a.q = q; a.beta = beta; a.rowsum = rowsum;
+  a.perm = nullptr; a.k = 1; a.interleave = 0;
+  return launch_quant_act(a, false, static_cast<cudaStream_t>(stream));
+}

@@ -1,0 +1,181 @@
+// Absmean ternary weight quantizer with INT2 packing (Eq. 7, 9, 10; storage per Section 3.1).
+//
+// Three launches per matrix:
+//   1. abs_sum_bins    exact accumulation of sum |w|: each fp32 magnitude is split into its
+//                      24-bit integer significand and its exponent; significands are added into
+//                      one 64-bit integer bin per exponent.  Integer adds commute, so the bins do
+//                      not depend on thread order.
+//   2. alpha_finalize  one thread adds the bins into a 384-bit integer (exact), rounds it to
+//                      fp64 (nearest even), divides by m*n in fp64 and rounds once to fp32.
+//   3. pack_codes      code = clamp(rint(w / alpha), -1, 1), four codes per byte.
+#include "mote_common.cuh"
+
+namespace mote {
+
+constexpr int kBins = 256;
+
+template <bool kBf16>
+__global__ void __launch_bounds__(256) abs_sum_bins_kernel(const void* __restrict__ W, int64_t n_vec,
+                                                           unsigned long long* __restrict__ bins) {
+  __shared__ unsigned long long sbins[kBins];
+  for (int i = threadIdx.x; i < kBins; i += blockDim.x) sbins[i] = 0ull;
+  __syncthreads();
+
+  const int lane = threadIdx.x & 31;
+  // one "vec" = 4 elements (a float4, or 4 bf16 = uint2)
+  const int64_t stride = int64_t(gridDim.x) * blockDim.x;
+  const int64_t first = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
+  // all lanes of a warp run the same number of iterations so the warp-wide votes stay converged
+  const int64_t warp_first = first - lane;
+  for (int64_t base = warp_first; base < n_vec; base += stride) {
+    const int64_t v = base + lane;
+    uint32_t bits[4] = {0u, 0u, 0u, 0u};
+    if (v < n_vec) {
+      if (kBf16) {
+        uint2 r = reinterpret_cast<const uint2*>(W)[v];
+        bits[0] = r.x << 16; bits[1] = r.x & 0xFFFF0000u; bits[2] = r.y << 16; bits[3] = r.y & 0xFFFF0000u;
+      } else {
+        uint4 r = reinterpret_cast<const uint4*>(W)[v];
+        bits[0] = r.x; bits[1] = r.y; bits[2] = r.z; bits[3] = r.w;
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const uint32_t a = bits[j] & 0x7FFFFFFFu;
+      const uint32_t e = a >> 23;
+      const uint32_t mant = e ? ((a & 0x7FFFFFu) | 0x800000u) : a;   // subnormals: no hidden bit
+      // lanes with the same exponent add their significands first (sum < 2^29)
+      const uint32_t peers = __match_any_sync(0xffffffffu, e);
+      const uint32_t sum = __reduce_add_sync(peers, mant);
+      if (lane == (__ffs(peers) - 1) && sum) atomicAdd(&sbins[e], (unsigned long long)sum);
+    }
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i < kBins; i += blockDim.x)
+    if (sbins[i]) atomicAdd(&bins[i], sbins[i]);
+}
+
+// bins[e] counts units of 2^(max(e,1) - 150).  total = sum_e bins[e] << (max(e,1) - 1) in units
+// of 2^-149.
+__global__ void alpha_finalize_kernel(const unsigned long long* __restrict__ bins, double count,
+                                      float* __restrict__ alpha) {
+  if (threadIdx.x != 0 || blockIdx.x != 0) return;
+  constexpr int kLimbs = 12;
+  uint32_t L[kLimbs];
+  for (int i = 0; i < kLimbs; ++i) L[i] = 0u;
+  for (int e = 0; e < 255; ++e) {            // e = 255 (inf/nan) is undefined input, ignored
+    const unsigned long long v = bins[e];
+    if (!v) continue;
+    const int s = (e ? e : 1) - 1;
+    const int wo = s >> 5, bo = s & 31;
+    const unsigned __int128 sv = (unsigned __int128)v << bo;   // < 2^95
+    uint32_t part[3] = {(uint32_t)sv, (uint32_t)(sv >> 32), (uint32_t)(sv >> 64)};
+    unsigned long long carry = 0ull;
+    for (int i = 0; i < 3; ++i) {
+      unsigned long long t = (unsigned long long)L[wo + i] + part[i] + carry;
+      L[wo + i] = (uint32_t)t;
+      carry = t >> 32;
+    }
+    for (int i = wo + 3; carry && i < kLimbs; ++i) {
+      unsigned long long t = (unsigned long long)L[i] + carry;
+      L[i] = (uint32_t)t;
+      carry = t >> 32;
+    }
+  }
+  int top = kLimbs - 1;
+  while (top >= 0 && L[top] == 0u) --top;
+  double sum = 0.0;
+  if (top >= 0) {
+    const int msb = top * 32 + (31 - __clz(L[top]));
+    auto bit = [&](int i) -> unsigned long long { return i < 0 ? 0ull : ((L[i >> 5] >> (i & 31)) & 1u); };
+    if (msb <= 52) {
+      unsigned long long m = 0ull;
+      for (int i = msb; i >= 0; --i) m = (m << 1) | bit(i);
+      sum = scalbn((double)m, -149);
+    } else {
+      const int sh = msb - 52;
+      unsigned long long m = 0ull;
+      for (int i = msb; i >= sh; --i) m = (m << 1) | bit(i);
+      const unsigned long long round_bit = bit(sh - 1);
+      unsigned long long sticky = 0ull;
+      for (int i = sh - 2; i >= 0 && !sticky; --i) sticky |= bit(i);
+      if (round_bit && (sticky || (m & 1ull))) ++m;     // nearest, ties to even
+      sum = scalbn((double)m, sh - 149);
+    }
+  }
+  const float a = (float)(sum / count);                  // fp64 divide, one rounding to fp32
+  *alpha = fmaxf(a, kEpsScale);
+}
+
+template <bool kBf16>
+__global__ void __launch_bounds__(256) pack_codes_kernel(const void* __restrict__ W, int64_t n_words,
+                                                         const float* __restrict__ alpha_ptr,
+                                                         uint32_t* __restrict__ packed) {
+  const float alpha = *alpha_ptr;
+  const int64_t stride = int64_t(gridDim.x) * blockDim.x;
+  for (int64_t w = int64_t(blockIdx.x) * blockDim.x + threadIdx.x; w < n_words; w += stride) {
+    float v[16];
+    if (kBf16) {
+      const uint4* src = reinterpret_cast<const uint4*>(W) + w * 2;
+#pragma unroll
+      for (int i = 0; i < 2; ++i) {
+        uint4 r = src[i];
+        uint32_t u[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) { v[i * 8 + 2 * j] = bf16_lo(u[j]); v[i * 8 + 2 * j + 1] = bf16_hi(u[j]); }
+      }
+    } else {
+      const float4* src = reinterpret_cast<const float4*>(W) + w * 4;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        float4 r = src[i];
+        v[4 * i] = r.x; v[4 * i + 1] = r.y; v[4 * i + 2] = r.z; v[4 * i + 3] = r.w;
+      }
+    }
+    uint32_t out = 0u;
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      float c = rintf(__fdiv_rn(v[j], alpha));
+      c = fminf(fmaxf(c, -1.0f), 1.0f);
+      out |= uint32_t(__float2int_rn(c) + 1) << (2 * j);
+    }
+    packed[w] = out;
+  }
+}
+
+}  // namespace mote
+
+extern "C" size_t mote_ternarize_workspace_bytes(void) { return mote::kBins * sizeof(unsigned long long); }
+
+extern "C" mote_status_t mote_ternarize_pack(const void* W, int w_dtype, int64_t m, int64_t n,
+                                             uint8_t* packed, float* alpha, void* ws, size_t ws_bytes,
+                                             void* stream_) {
+  using namespace mote;
+  if (!W || !packed || !alpha || !ws) return MOTE_ERR_NULL;
+  if (w_dtype != MOTE_DTYPE_F32 && w_dtype != MOTE_DTYPE_BF16) return MOTE_ERR_DTYPE;
+  if (m <= 0 || n <= 0 || (n % 16) != 0) return MOTE_ERR_SHAPE;
+  if (m >= (int64_t(1) << 38) / n) return MOTE_ERR_SHAPE;
+  if (!aligned16(W) || !aligned16(packed) || !aligned16(ws)) return MOTE_ERR_ALIGN;
+  if (ws_bytes < mote_ternarize_workspace_bytes()) return MOTE_ERR_WORKSPACE;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  auto* bins = static_cast<unsigned long long*>(ws);
+  const int64_t total = m * n;
+  const int64_t n_vec = total / 4, n_words = total / 16;
+  MOTE_CUDA_OK(cudaMemsetAsync(bins, 0, mote_ternarize_workspace_bytes(), stream));
+  const int threads = 256;
+  int blocks_a = (int)std::min<int64_t>((n_vec + threads - 1) / threads, 148 * 8);
+  int blocks_c = (int)std::min<int64_t>((n_words + threads - 1) / threads, 148 * 16);
+  if (w_dtype == MOTE_DTYPE_BF16)
+    abs_sum_bins_kernel<true><<<blocks_a, threads, 0, stream>>>(W, n_vec, bins);
+  else
+    abs_sum_bins_kernel<false><<<blocks_a, threads, 0, stream>>>(W, n_vec, bins);
+  MOTE_LAUNCH_OK();
+  alpha_finalize_kernel<<<1, 32, 0, stream>>>(bins, (double)total, alpha);
+  MOTE_LAUNCH_OK();
+  if (w_dtype == MOTE_DTYPE_BF16)
+    pack_codes_kernel<true><<<blocks_c, threads, 0, stream>>>(W, n_words, alpha, reinterpret_cast<uint32_t*>(packed));
+  else
+    pack_codes_kernel<false><<<blocks_c, threads, 0, stream>>>(W, n_words, alpha, reinterpret_cast<uint32_t*>(packed));
+  MOTE_LAUNCH_OK();
+  return MOTE_OK;
+}

@@ -1,0 +1,78 @@
+"""Helpers for the GPU parity tests: run the library through its C ABI on seeded inputs and
+compare every intermediate with the CPU oracle."""
+import numpy as np
+import torch
+
+from oracle import mote_oracle as O
+
+REL_FRO_TOL = 5e-3      # bf16 layer output against the fp64 oracle
+GATE_W_TOL = 1e-6
+
+
+def bf16_tensor(bits: np.ndarray, device="cuda") -> torch.Tensor:
+    return torch.from_numpy(bits.view(np.int16).copy()).view(torch.bfloat16).to(device)
+
+
+def bf16_bits(t: torch.Tensor) -> np.ndarray:
+    return t.detach().cpu().contiguous().view(torch.int16).numpy().view(np.uint16)
+
+
+def oracle_layer_from_master(master: dict) -> dict:
+    return O.build_layer(master)
+
+
+def check_packed_layer(layer_gpu, layer_or: dict):
+    """Packed bytes and alpha of every routed matrix: bit-exact."""
+    for name in ("gate", "up", "down"):
+        packed = layer_gpu.tensors[name + "_packed"].cpu().numpy()
+        alpha = layer_gpu.tensors["alpha_" + name].cpu().numpy()
+        for e in range(layer_or["E"]):
+            want = O.pack_codes(layer_or["codes_" + name][e])
+            assert np.array_equal(packed[e], want), (name, e)
+            assert alpha[e] == layer_or["alpha_" + name][e], (name, e, alpha[e], layer_or["alpha_" + name][e])
+
+
+def check_forward(mote, layer_gpu, layer_or: dict, x_bits: np.ndarray, residual_bits=None, token_subset=None,
+                  out_alias_residual=False):
+    """Runs mote_moe_forward with every tap and compares with the oracle.  Returns a report."""
+    T, d = x_bits.shape
+    k, E, f = layer_or["k"], layer_or["E"], layer_or["f"]
+    x = bf16_tensor(x_bits)
+    res = None if residual_bits is None else bf16_tensor(residual_bits)
+    taps = layer_gpu.alloc_taps(T)
+    out_buf = res if out_alias_residual else None
+    out = mote.mote_moe_forward(layer_gpu, x, residual=res, out=out_buf, taps=taps)
+    torch.cuda.synchronize()
+    g = {n: t.cpu() for n, t in taps.items()}
+    g_idx = g["topk_idx"].numpy()
+
+    ref = O.moe_forward(layer_or, x_bits, residual_bits, token_subset=token_subset, near_tie_choice=g_idx)
+    near = ref["near_tie"]
+    # routing: indices equal everywhere (near-tie tokens were aligned to the GPU's valid choice)
+    for t in np.nonzero(near)[0]:
+        top = np.sort(ref["logits"][t])[::-1]
+        assert set(g_idx[t]) <= set(np.nonzero(ref["logits"][t] >= top[k - 1] - 1e-5 - 1e-12)[0].tolist())
+    assert np.array_equal(g_idx, ref["topk_idx"])
+    assert np.max(np.abs(g["topk_w"].numpy().astype(np.float64) - ref["topk_w"])) <= GATE_W_TOL
+    assert np.array_equal(g["offsets"].numpy(), ref["offsets"])
+    assert np.array_equal(g["perm"].numpy(), ref["perm"])
+    assert np.array_equal(g["qx"].numpy(), ref["qx"])
+    assert np.array_equal(g["beta_x"].numpy(), ref["beta_x"])
+    rows = ref["rows"]
+    assert np.array_equal(g["acc_gate"].numpy()[rows], ref["acc_gate"])
+    assert np.array_equal(g["acc_up"].numpy()[rows], ref["acc_up"])
+    assert np.array_equal(bf16_bits(g["h_bf16"])[rows], ref["h_bf16"])
+    assert np.array_equal(g["qh"].numpy()[rows], ref["qh"])
+    assert np.array_equal(g["beta_h"].numpy()[rows], ref["beta_h"])
+    assert np.array_equal(g["acc_down"].numpy()[rows], ref["acc_down"])
+    y = g["y"].numpy()[rows].astype(np.float64)
+    assert np.allclose(y, ref["y"], rtol=2e-6, atol=1e-12)
+    toks = ref["tokens"]
+    sh = g["shared_out"].numpy()[toks].astype(np.float64)
+    sh_err = np.linalg.norm(sh - ref["shared_out"]) / max(np.linalg.norm(ref["shared_out"]), 1e-30)
+    assert sh_err <= REL_FRO_TOL, sh_err
+    out_f = O.bf16_to_f32(bf16_bits(out))[toks].astype(np.float64)
+    err = np.linalg.norm(out_f - ref["out"]) / max(np.linalg.norm(ref["out"]), 1e-30)
+    assert err <= REL_FRO_TOL, err
+    return dict(rel_fro=err, shared_rel_fro=sh_err, near_ties=int(near.sum()), tokens=len(toks),
+                out=out, counts=np.diff(ref["offsets"]))

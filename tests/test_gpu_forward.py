@@ -1,0 +1,110 @@
+"""GPU parity of the whole layer (mote_moe_forward through the C ABI) against the CPU oracle:
+every integer stage bit-exact, the bf16 output within 5e-3 relative Frobenius error."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import mote_oracle as O
+from workloads import synth
+from tests.parity_utils import bf16_bits, bf16_tensor, check_forward, check_packed_layer
+
+pytestmark = pytest.mark.gpu
+
+PATHS = {"simt": 1}
+
+
+@pytest.fixture(scope="module")
+def mote():
+    import paper_2506_14435_b200 as m
+    return m
+
+
+def _setup(mote, wl, path=1):
+    master = synth.master_layer(wl)
+    layer_or = O.build_layer(master)
+    layer_gpu = mote.MoteLayer.from_master(master, path=path)
+    return master, layer_or, layer_gpu
+
+
+def test_c1_full_parity(mote):
+    wl = synth.WORKLOADS["c1"]
+    master, layer_or, layer_gpu = _setup(mote, wl)
+    check_packed_layer(layer_gpu, layer_or)
+    rep = check_forward(mote, layer_gpu, layer_or, synth.tokens(wl))
+    assert rep["rel_fro"] < 5e-3
+
+
+@pytest.mark.parametrize("d,f,E,k,T,kw", [
+    (16, 32, 3, 2, 5, {}),
+    (48, 80, 2, 1, 1, {}),
+    (64, 112, 5, 5, 33, {}),                       # k = E
+    (256, 512, 4, 2, 300, dict(outlier_frac=0.02)),
+    (128, 256, 8, 2, 77, dict(bias="zipf")),
+    (128, 384, 4, 1, 130, dict(norm_topk=0)),
+])
+def test_small_shapes(mote, d, f, E, k, T, kw):
+    wl = synth.custom("small", d, f, E, k, T, 2000 + d + f + T, **kw)
+    master, layer_or, layer_gpu = _setup(mote, wl)
+    check_packed_layer(layer_gpu, layer_or)
+    check_forward(mote, layer_gpu, layer_or, synth.tokens(wl))
+
+
+def test_idle_and_overloaded_experts_residual_and_aliasing(mote):
+    wl = synth.custom("skew", 128, 256, 4, 2, 97, 3001)
+    master = synth.master_layer(wl)
+    master["router_bias"] = np.array([50.0, -50.0, 40.0, -60.0], np.float32)   # experts 1 and 3 idle
+    layer_or = O.build_layer(master)
+    layer_gpu = mote.MoteLayer.from_master(master, path=1)
+    x = synth.tokens(wl)
+    res = synth.tokens(wl, stream=1)
+    rep = check_forward(mote, layer_gpu, layer_or, x, residual_bits=res)
+    assert rep["counts"].tolist() == [97, 0, 97, 0]
+    rep2 = check_forward(mote, layer_gpu, layer_or, x, residual_bits=res, out_alias_residual=True)
+    assert torch.equal(rep["out"], rep2["out"])
+
+
+def test_run_to_run_determinism_and_token_permutation(mote):
+    wl = synth.custom("det", 256, 512, 4, 2, 200, 3002)
+    master, layer_or, layer_gpu = _setup(mote, wl)
+    x = bf16_tensor(synth.tokens(wl))
+    a = mote.mote_moe_forward(layer_gpu, x).clone()
+    b = mote.mote_moe_forward(layer_gpu, x).clone()
+    assert torch.equal(a, b)
+    pm = torch.randperm(wl.T, generator=torch.Generator().manual_seed(1)).cuda()
+    c = mote.mote_moe_forward(layer_gpu, x[pm].contiguous())
+    assert torch.equal(c, a[pm])
+
+
+def test_zero_tokens_is_a_noop(mote):
+    wl = synth.WORKLOADS["c1"]
+    master, layer_or, layer_gpu = _setup(mote, wl)
+    x = torch.empty((0, wl.d), dtype=torch.bfloat16, device="cuda")
+    out = mote.mote_moe_forward(layer_gpu, x)
+    assert out.shape == (0, wl.d)
+
+
+@pytest.mark.parametrize("T", synth.C3_BATCHES)
+def test_c3_decode_batches(mote, T, c3_layers):
+    wl, layer_or, layer_gpu = c3_layers
+    rep = check_forward(mote, layer_gpu, layer_or, synth.tokens(wl, T=T))
+    assert rep["rel_fro"] < 5e-3
+
+
+@pytest.fixture(scope="module")
+def c3_layers(mote):
+    wl = synth.WORKLOADS["c3"]
+    master, layer_or, layer_gpu = _setup(mote, wl)
+    check_packed_layer(layer_gpu, layer_or)
+    return wl, layer_or, layer_gpu
+
+
+def test_host_buffer_entry_point(mote):
+    from paper_2506_14435_b200.binding import mote_moe_forward_host
+    wl = synth.WORKLOADS["c1"]
+    master, layer_or, layer_gpu = _setup(mote, wl)
+    xb = synth.tokens(wl)
+    x_host = torch.from_numpy(xb.view(np.int16).copy()).view(torch.bfloat16).pin_memory()
+    out_host = torch.empty_like(x_host).pin_memory()
+    mote_moe_forward_host(layer_gpu, x_host, out_host)
+    want = mote.mote_moe_forward(layer_gpu, x_host.cuda())
+    assert torch.equal(out_host, want.cpu())

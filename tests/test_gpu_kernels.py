@@ -1,0 +1,116 @@
+"""GPU parity of the three stand-alone entry points against the CPU oracle (bit-exact integer
+stages, gate weights within 1e-6)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import mote_oracle as O
+from workloads import synth
+from tests.parity_utils import bf16_bits, bf16_tensor
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def mote():
+    import paper_2506_14435_b200 as m
+    return m
+
+
+def _randn(shape, seed, scale=1.0):
+    return (torch.randn(shape, generator=torch.Generator().manual_seed(seed)) * scale).numpy()
+
+
+@pytest.mark.parametrize("m,n,scale", [(1, 16, 0.02), (7, 48, 0.02), (256, 512, 0.02), (300, 1008, 1.0),
+                                       (4864, 896, 0.02), (129, 11008, 0.02), (64, 64, 1e-30), (64, 64, 1e30)])
+def test_ternarize_pack_fp32(mote, m, n, scale):
+    W = _randn((m, n), 100 + m + n, scale).astype(np.float32)
+    codes, alpha = O.ternarize(W)
+    packed, a = mote.mote_ternarize_pack(torch.from_numpy(W).cuda())
+    assert a.item() == alpha
+    assert np.array_equal(packed.cpu().numpy(), O.pack_codes(codes))
+
+
+def test_ternarize_pack_special_values(mote):
+    W = np.zeros((8, 32), np.float32)
+    packed, a = mote.mote_ternarize_pack(torch.from_numpy(W).cuda())
+    assert a.item() == np.float32(1e-5) and np.all(packed.cpu().numpy() == 0x55)
+    # exact ties at +-0.5 and +-1.5 of alpha, subnormals, wide exponent spread
+    W = np.tile(np.array([0.5, -0.5, 1.5, -1.5, 1.0, -1.0, 1.0, 1.0], np.float32), (4, 4))
+    codes, alpha = O.ternarize(W)
+    packed, a = mote.mote_ternarize_pack(torch.from_numpy(W).cuda())
+    assert a.item() == alpha == 1.0 and np.array_equal(packed.cpu().numpy(), O.pack_codes(codes))
+    rng = np.random.default_rng(3)
+    W = (rng.standard_normal((64, 256)) * np.exp2(rng.integers(-140, 60, size=(64, 256)))).astype(np.float32)
+    codes, alpha = O.ternarize(W)
+    packed, a = mote.mote_ternarize_pack(torch.from_numpy(W).cuda())
+    assert a.item() == alpha and np.array_equal(packed.cpu().numpy(), O.pack_codes(codes))
+
+
+def test_ternarize_pack_bf16_input(mote):
+    Wb = O.f32_to_bf16_rn(_randn((96, 320), 5, 0.02).astype(np.float32))
+    codes, alpha = O.ternarize(O.bf16_to_f32(Wb))
+    packed, a = mote.mote_ternarize_pack(bf16_tensor(Wb))
+    assert a.item() == alpha and np.array_equal(packed.cpu().numpy(), O.pack_codes(codes))
+
+
+@pytest.mark.parametrize("T,d", [(1, 16), (5, 48), (64, 256), (300, 896), (33, 1536), (17, 2048), (9, 4864),
+                                 (6, 8960), (5, 11008), (3, 32768)])
+def test_quant_act(mote, T, d):
+    x = O.f32_to_bf16_rn(_randn((T, d), 7 * T + d, 3.0).astype(np.float32))
+    if T > 2:
+        x[1] = 0
+        x[2, : d // 2] = 0
+    q, beta, rowsum = O.quant_act(x)
+    gq, gb, gs = mote.mote_quant_act(bf16_tensor(x))
+    assert np.array_equal(gq.cpu().numpy(), q)
+    assert np.array_equal(gb.cpu().numpy(), beta)
+    assert np.array_equal(gs.cpu().numpy(), rowsum)
+
+
+def test_quant_act_strided_rows_and_outliers(mote):
+    wl = synth.WORKLOADS["c2"]
+    x = synth.tokens(wl, T=200)
+    wide = np.zeros((200, wl.d + 64), np.uint16)
+    wide[:, : wl.d] = x
+    xt = bf16_tensor(wide)[:, : wl.d]
+    q, beta, rowsum = O.quant_act(x)
+    gq, gb, gs = mote.mote_quant_act(xt)
+    assert np.array_equal(gq.cpu().numpy(), q) and np.array_equal(gb.cpu().numpy(), beta)
+    assert np.array_equal(gs.cpu().numpy(), rowsum)
+    assert gq.abs().max().item() == 127
+
+
+@pytest.mark.parametrize("name,T,k,norm", [("c1", 64, 2, 1), ("c1", 64, 1, 0), ("c1", 64, 4, 0), ("c3", 64, 2, 1),
+                                           ("c3", 1, 2, 1), ("c4", 1000, 2, 1), ("c4", 257, 8, 0)])
+def test_route_topk(mote, name, T, k, norm):
+    wl = synth.WORKLOADS[name]
+    x = synth.tokens(wl, T=T)
+    Wr, bias = synth.router_weights(wl, 0)
+    ref = O.router(x, Wr, bias, k, norm)
+    idx, w, logits = mote.mote_route_topk(bf16_tensor(x), torch.from_numpy(Wr).cuda(),
+                                          None if bias is None else torch.from_numpy(bias).cuda(), k, norm,
+                                          want_logits=True)
+    idx, w, logits = idx.cpu().numpy(), w.cpu().numpy(), logits.cpu().numpy()
+    assert np.max(np.abs(logits - ref["logits"])) < 2e-5
+    ok = ~ref["near_tie"]
+    assert np.array_equal(idx[ok], ref["idx"][ok])
+    assert np.max(np.abs(w[ok].astype(np.float64) - ref["w"][ok])) <= 1e-6
+    if norm:
+        assert np.allclose(w.sum(axis=1), 1.0, atol=1e-6)
+
+
+def test_route_topk_many_experts_and_ties(mote):
+    rng = np.random.default_rng(11)
+    T, d, E = 50, 64, 64
+    x = O.f32_to_bf16_rn(rng.standard_normal((T, d)).astype(np.float32))
+    Wr = O.bf16_to_f32(O.f32_to_bf16_rn((rng.standard_normal((E, d)) * 0.1).astype(np.float32)))
+    Wr[40] = Wr[3]                                   # an exact tie: the lower index must win
+    ref = O.router(x, Wr, None, 8, 1)
+    idx, w, _ = mote.mote_route_topk(bf16_tensor(x), torch.from_numpy(Wr).cuda(), None, 8, 1)
+    idx = idx.cpu().numpy()
+    for t in range(T):
+        if 3 in idx[t] and 40 in idx[t]:
+            assert list(idx[t]).index(3) < list(idx[t]).index(40)
+    ok = ~ref["near_tie"]
+    assert np.array_equal(idx[ok], ref["idx"][ok])
