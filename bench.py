@@ -1,0 +1,316 @@
+#!/usr/bin/env python
+"""Benchmark of the MoTE FFN-layer forward pass on B200.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2|c4|c3-T|c1] [--impl ours|reference]
+
+One "step" is one pass of the whole layer (route, dispatch, Q_a(x), gate/up ternary GEMM, Q_a(h),
+down ternary GEMM, shared bf16 FFN, combine) over one batch of synthetic tokens.  Weights are
+ternarized once, before the timed region (offline step).  Prints ONE JSON line.
+
+Multi-GPU: the layer is token-parallel with no exchange step, so every rank holds a full replica
+and its own batch (weak scaling, no collective on the data path); the job value is the sum of the
+ranks' tokens over the slowest rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from workloads import synth  # noqa: E402
+
+L2_FLUSH_BYTES = 512 << 20
+NOMINAL_INT8_OVER_BF16 = 2.0      # dense tensor peak ratio int8 : bf16 (4.5 vs 2.25 POP/s nominal)
+
+
+def parse_workload(name: str) -> synth.Workload:
+    if name.startswith("c3-"):
+        return synth.WORKLOADS["c3"].with_T(int(name[3:]))
+    if name.startswith("c5-"):
+        return synth.WORKLOADS["c5"].with_T(int(name[3:]))
+    return synth.WORKLOADS[name]
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm_gbs=p["hbm_gbs"], bf16_tflops=p["bf16_tflops"],
+                    bf16_tflops_sustained=p.get("bf16_tflops_sustained", p["bf16_tflops"]), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.12)
+        self.proc.terminate()
+        self.thread.join(timeout=2)
+        sm, mx, reasons = [], None, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            p = [s.strip() for s in ln.split(",")]
+            if len(p) < 6:
+                continue
+            try:
+                sm.append(float(p[0])); mx = float(p[1])
+            except ValueError:
+                continue
+            for n, v in zip(names, p[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def build_gpu_layer(wl: synth.Workload, device):
+    import paper_2506_14435_b200 as mote
+    master = synth.master_layer(wl)
+    return mote, mote.MoteLayer.from_master(master, device=device), master
+
+
+def dominant_stage_work(wl: synth.Workload, stage: str, counts=None):
+    """Algorithmic work of one launch of a stage: (amount, kind) with kind 'int8' | 'bf16' | 'bytes'."""
+    P, T, d, f = wl.T * wl.k, wl.T, wl.d, wl.f
+    if stage == "gateup_ternary":
+        return 2.0 * P * d * 2 * f, "int8"
+    if stage == "down_ternary":
+        return 2.0 * P * f * d, "int8"
+    if stage == "shared_gateup":
+        return 2.0 * T * d * 2 * f, "bf16"
+    if stage == "shared_down":
+        return 2.0 * T * f * d, "bf16"
+    if stage == "quant_x":
+        return T * d * 2.0 + P * d * 1.0, "bytes"
+    if stage == "quant_h":
+        return P * f * 3.0, "bytes"
+    if stage == "combine":
+        return T * d * (4.0 + 4.0 * wl.k + 2.0), "bytes"
+    if stage == "route":
+        return T * d * 2.0, "bytes"
+    return P * 12.0, "bytes"
+
+
+def run_ours(args):
+    rank = int(os.environ.get("RANK", 0))
+    local_rank = int(os.environ.get("LOCAL_RANK", 0))
+    world = int(os.environ.get("WORLD_SIZE", 1))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback for the product path")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    wl = parse_workload(args.workload)
+    mote, layer, master = build_gpu_layer(wl, dev)
+    from paper_2506_14435_b200.binding import mote_moe_forward_host, mote_moe_forward_profile
+
+    x_bits = synth.tokens(wl, stream=rank)
+    x_host = torch.from_numpy(x_bits.view(np.int16).copy()).view(torch.bfloat16).pin_memory()
+    out_host = torch.empty_like(x_host).pin_memory()
+    x = x_host.to(dev)
+    out = torch.empty_like(x)
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed_loop(step_fn, n):
+        starts = [torch.cuda.Event(enable_timing=True) for _ in range(n)]
+        ends = [torch.cuda.Event(enable_timing=True) for _ in range(n)]
+        for i in range(n):
+            flush.fill_(i & 0xFF)                       # evict L2 between iterations
+            starts[i].record(stream)
+            step_fn()
+            ends[i].record(stream)
+        torch.cuda.synchronize()
+        return [s.elapsed_time(e) for s, e in zip(starts, ends)]
+
+    # ---- device-resident timing
+    for _ in range(args.warmup):
+        mote.mote_moe_forward(layer, x, out=out)
+    launches_per_step = mote.lib.mote_last_launch_count()
+    barrier()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    per_step = timed_loop(lambda: mote.mote_moe_forward(layer, x, out=out), args.steps)
+    barrier()
+    total_ms = sum(per_step)
+
+    # ---- per-stage device times of the same launch configuration (events on the launch stream)
+    stage_acc = {}
+    n_prof = max(3, min(args.steps, 10))
+    for i in range(n_prof):
+        flush.fill_(i)
+        ms = mote_moe_forward_profile(layer, x, out=out)
+        for k_, v in ms.items():
+            stage_acc.setdefault(k_, []).append(v)
+    clocks = sampler.stop() if rank == 0 else None
+    stage_ms = {k_: statistics.mean(v) for k_, v in stage_acc.items()}
+
+    # ---- end to end through the host-buffer entry point
+    for _ in range(min(args.warmup, 3)):
+        mote_moe_forward_host(layer, x_host, out_host)
+    barrier()
+    e2e_ms = []
+    for i in range(args.steps):
+        flush.fill_(i & 0xFF)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        mote_moe_forward_host(layer, x_host, out_host)      # synchronises the stream itself
+        e2e_ms.append((time.perf_counter() - t0) * 1e3)
+    barrier()
+    e2e_total = sum(e2e_ms)
+
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([total_ms, e2e_total], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms, e2e_total = t.tolist()
+    if rank != 0:
+        if world > 1:
+            import torch.distributed as dist
+            dist.destroy_process_group()
+        return
+
+    peaks = measured_peaks()
+    ms_per_step = total_ms / args.steps
+    tokens_per_s = world * wl.T * args.steps / (total_ms * 1e-3)
+    decode = wl.T <= 64
+    dom = max(stage_ms, key=stage_ms.get)
+    work, kind = dominant_stage_work(wl, dom)
+    dur_s = stage_ms[dom] * 1e-3
+    if kind == "bytes":
+        roof = dict(bound="hbm", achieved=work / dur_s / 1e9, peak=peaks["hbm_gbs"], unit="GB/s")
+    else:
+        peak = peaks["bf16_tflops"] * (NOMINAL_INT8_OVER_BF16 if kind == "int8" else 1.0)
+        roof = dict(bound="tensor", achieved=work / dur_s / 1e12, peak=peak, unit="TOP/s" if kind == "int8" else "TFLOP/s")
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    roof["traffic"] = None
+    roof["kernel"] = dom
+    roof["kernel_ms"] = stage_ms[dom]
+    roof["peak_source"] = ("of measured" if peaks["source"] == "measured" else "of fallback") + \
+        (" (bf16 burst x2 nominal int8:bf16 ratio)" if kind == "int8" else "")
+
+    line = {
+        "metric": "MoTE layer tokens/sec (prefill)" if not decode else "MoTE layer tokens/sec (decode batch)",
+        "value": tokens_per_s, "unit": "tokens/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "us_per_layer": ms_per_step * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "int8xint2->int32 routed, bf16 shared", "data": "synthetic",
+        "config": {"workload": wl.name, "d": wl.d, "f": wl.f, "E": wl.E, "k": wl.k, "T_per_gpu": wl.T,
+                   "l2": "flushed between timed iterations (512 MiB write)", "parallelism": f"replicas x{world}"},
+        "stage_ms": stage_ms, "roofline": roof,
+        "e2e": {"value": world * wl.T * args.steps / (e2e_total * 1e-3), "unit": "tokens/s",
+                "h2d_bytes_per_step": int(x_host.numel() * 2), "d2h_bytes_per_step": int(out_host.numel() * 2)},
+        "gpu_launches": launches_per_step * args.steps, "clocks": clocks,
+    }
+    if world == 1:
+        line["cpu_baseline"] = cpu_baseline(wl, master, x_bits, budget_s=20.0)
+    print(json.dumps(line))
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+def cpu_baseline(wl, master, x_bits, budget_s: float, n_tokens: int | None = None):
+    """The oracle as it stands, on the host cores, on a bounded sample of the same workload."""
+    from oracle import mote_oracle as O
+    layer_or = O.build_layer(master)                     # offline step, not timed (as on the GPU)
+    n = n_tokens or min(wl.T, 256 if wl.d * wl.f < 8e6 else 64)
+    sub = np.arange(n)
+    t0 = time.perf_counter()
+    O.moe_forward(layer_or, x_bits, token_subset=sub)
+    dt = time.perf_counter() - t0
+    return {"value": n / dt, "unit": "tokens/s", "cores": torch.get_num_threads(), "kind": "oracle",
+            "sample": f"first {n} of {wl.T} tokens of {wl.name} (routing for all tokens), {dt:.2f} s",
+            "seconds": dt}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", 0))
+    if rank != 0:
+        return
+    wl = parse_workload(args.workload)
+    master = synth.master_layer(wl)
+    from oracle import mote_oracle as O
+    layer_or = O.build_layer(master)
+    x_bits = synth.tokens(wl)
+    n = min(wl.T, 128 if wl.d * wl.f < 8e6 else 32)
+    sub = np.arange(n)
+    for _ in range(args.warmup):
+        O.moe_forward(layer_or, x_bits, token_subset=sub)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        O.moe_forward(layer_or, x_bits, token_subset=sub)
+    dt = time.perf_counter() - t0
+    val = n * args.steps / dt
+    decode = wl.T <= 64
+    print(json.dumps({
+        "impl": "reference",
+        "metric": "MoTE layer tokens/sec (prefill)" if not decode else "MoTE layer tokens/sec (decode batch)",
+        "value": val, "unit": "tokens/s", "n_gpus": int(os.environ.get("WORLD_SIZE", 1)), "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "fp64 / exact integers", "data": "synthetic",
+        "config": {"workload": wl.name, "d": wl.d, "f": wl.f, "E": wl.E, "k": wl.k, "T_per_gpu": wl.T},
+        "cpu_baseline": {"value": val, "unit": "tokens/s", "cores": torch.get_num_threads(), "kind": "oracle",
+                         "sample": f"each step = first {n} of {wl.T} tokens of {wl.name}"},
+        "e2e": {"value": val, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="c2")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

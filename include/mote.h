@@ -171,6 +171,17 @@ mote_status_t mote_moe_forward_host(const mote_layer_t* L, const void* x_host,
                                     const void* residual_host, int64_t T, void* out_host,
                                     void* ws, size_t ws_bytes, void* stream);
 
+/* mote_moe_forward with a CUDA event recorded on `stream` between the stages; waits for the stream
+ * and writes the device time of each stage, in milliseconds, to stage_ms_host[MOTE_N_STAGES]:
+ *   0 route (Eq. 3)   1 dispatch   2 Q_a(x) (Eq. 8)   3 gate/up ternary GEMM (Eq. 6)   4 Q_a(h)
+ *   5 down ternary GEMM (Eq. 5)   6 shared gate/up   7 shared down (Eq. 2)   8 combine (Eq. 2, 4)
+ * A stage that a fused path folds into its neighbour reports 0.  Stages run back to back on one
+ * stream here even if mote_moe_forward overlaps some of them. */
+enum { MOTE_N_STAGES = 9 };
+mote_status_t mote_moe_forward_profile(const mote_layer_t* L, const void* x_bf16,
+                                       const void* residual_bf16, int64_t T, void* out_bf16,
+                                       void* ws, size_t ws_bytes, void* stream, float* stage_ms_host);
+
 /* Reads (and clears) the device status word kept at the start of a workspace after the stream has
  * been synchronised by the caller: MOTE_OK, or MOTE_ERR_DEVICE_TIMEOUT if a kernel gave up a
  * bounded wait.  Synchronises the stream itself. */

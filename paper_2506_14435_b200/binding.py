@@ -58,6 +58,9 @@ lib.mote_moe_forward.argtypes = [C.POINTER(mote_layer_t), C.c_void_p, C.c_void_p
 lib.mote_moe_forward_host.restype = C.c_int
 lib.mote_moe_forward_host.argtypes = [C.POINTER(mote_layer_t), C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p,
                                       C.c_void_p, C.c_size_t, C.c_void_p]
+lib.mote_moe_forward_profile.restype = C.c_int
+lib.mote_moe_forward_profile.argtypes = [C.POINTER(mote_layer_t), C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p,
+                                         C.c_void_p, C.c_size_t, C.c_void_p, C.POINTER(C.c_float)]
 lib.mote_device_status.restype = C.c_int
 lib.mote_device_status.argtypes = [C.c_void_p, C.c_void_p]
 lib.mote_last_launch_count.restype = C.c_int
@@ -225,3 +228,21 @@ def mote_moe_forward_host(layer: MoteLayer, x_host: torch.Tensor, out_host: torc
     _check(lib.mote_moe_forward_host(C.byref(s), _ptr(x_host), _ptr(residual_host), T, _ptr(out_host), _ptr(ws),
                                      ws.numel(), _stream()), "mote_moe_forward_host")
     return out_host
+
+
+STAGE_NAMES = ["route", "dispatch", "quant_x", "gateup_ternary", "quant_h", "down_ternary", "shared_gateup",
+               "shared_down", "combine"]
+
+
+def mote_moe_forward_profile(layer: MoteLayer, x: torch.Tensor, out=None, residual=None) -> dict:
+    """One forward with CUDA events between the stages; returns {stage: milliseconds}."""
+    _need_cuda(x, residual, out)
+    T = x.shape[0]
+    if out is None:
+        out = torch.empty_like(x)
+    ws = layer.workspace(T)
+    s = layer.struct()
+    ms = (C.c_float * len(STAGE_NAMES))()
+    _check(lib.mote_moe_forward_profile(C.byref(s), _ptr(x), _ptr(residual), T, _ptr(out), _ptr(ws), ws.numel(),
+                                        _stream(), ms), "mote_moe_forward_profile")
+    return dict(zip(STAGE_NAMES, [float(v) for v in ms]))

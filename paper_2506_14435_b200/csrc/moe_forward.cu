@@ -12,6 +12,17 @@ namespace mote {
 
 thread_local int g_launch_count = 0;
 
+// Optional per-stage CUDA events (mote_moe_forward_profile): event i is recorded on the launch
+// stream after stage i has been enqueued, event 0 before the first stage.
+struct StageTimer {
+  cudaEvent_t ev[MOTE_N_STAGES + 1];
+  bool active = false;
+};
+static thread_local StageTimer g_timer;
+static inline void stage_mark(int i, cudaStream_t stream) {
+  if (g_timer.active) cudaEventRecord(g_timer.ev[i], stream);
+}
+
 struct Plan {
   size_t status, topk_idx, topk_w, offsets, perm, inv;
   size_t qx, beta_x, rowsum_x, h, qh, beta_h, rowsum_h, y, hs, s;
@@ -167,17 +178,21 @@ extern "C" mote_status_t mote_moe_forward(const mote_layer_t* L, const void* x, 
   const int interleave = 0;
 
   mote_status_t st;
+  stage_mark(0, stream);
   // S1 router, S2 dispatch
   st = launch_route_topk(x, T, d, L->Wr, L->router_bias, E, k, L->norm_topk, topk_idx, topk_w, nullptr, stream);
   if (st) return st;
+  stage_mark(1, stream);
   st = launch_dispatch(topk_idx, P, E, offsets, perm, inv, stream);
   if (st) return st;
+  stage_mark(2, stream);
   // S3 Q_a(x), written once per selected expert into the expert-sorted rows
   QuantActArgs qa{};
   qa.x = x; qa.T = T; qa.d = d; qa.ldx = d; qa.q = qx; qa.beta = beta_x; qa.rowsum = rowsum_x;
   qa.perm = perm; qa.k = k; qa.interleave = interleave;
   st = launch_quant_act(qa, true, stream);
   if (st) return st;
+  stage_mark(3, stream);
   // S4 gate/up
   TernaryGemmArgs g1{};
   g1.qa = qx; g1.beta = beta_x; g1.offsets = offsets; g1.w0 = L->gate_packed; g1.w1 = L->up_packed;
@@ -185,26 +200,32 @@ extern "C" mote_status_t mote_moe_forward(const mote_layer_t* L, const void* x, 
   g1.h_bf16 = h; g1.acc0_tap = taps ? taps->acc_gate : nullptr; g1.acc1_tap = taps ? taps->acc_up : nullptr;
   st = launch_ternary_gateup_simt(g1, stream);
   if (st) return st;
+  stage_mark(4, stream);
   // S5 Q_a(h)
   QuantActArgs qb{};
   qb.x = h; qb.T = P; qb.d = f; qb.ldx = f; qb.q = qh; qb.beta = beta_h; qb.rowsum = rowsum_h;
   qb.perm = nullptr; qb.k = 1; qb.interleave = interleave;
   st = launch_quant_act(qb, false, stream);
   if (st) return st;
+  stage_mark(5, stream);
   // S6 down
   TernaryGemmArgs g2{};
   g2.qa = qh; g2.beta = beta_h; g2.offsets = offsets; g2.w0 = L->down_packed; g2.alpha0 = L->alpha_down;
   g2.E = E; g2.N = d; g2.K = f; g2.P = P; g2.y = y; g2.acc0_tap = taps ? taps->acc_down : nullptr;
   st = launch_ternary_down_simt(g2, stream);
   if (st) return st;
+  stage_mark(6, stream);
   // S7 shared expert
   st = launch_shared_gateup_simt(x, L->sh_gate, L->sh_up, T, d, f, hs, stream);
   if (st) return st;
+  stage_mark(7, stream);
   st = launch_shared_down_simt(hs, L->sh_down, T, d, f, s, stream);
   if (st) return st;
+  stage_mark(8, stream);
   // S8 combine
   st = launch_combine(s, y, topk_w, perm, residual, T, d, k, out, stream);
   if (st) return st;
+  stage_mark(9, stream);
 
   if (taps) {
     auto d2d = [&](void* dst, const void* src, size_t bytes) -> bool {
@@ -254,4 +275,23 @@ extern "C" mote_status_t mote_moe_forward_host(const mote_layer_t* L, const void
   MOTE_CUDA_OK(cudaMemcpyAsync(out_host, out_dev, bytes, cudaMemcpyDeviceToHost, stream));
   MOTE_CUDA_OK(cudaStreamSynchronize(stream));
   return MOTE_OK;
+}
+
+extern "C" mote_status_t mote_moe_forward_profile(const mote_layer_t* L, const void* x, const void* residual,
+                                                  int64_t T, void* out, void* ws, size_t ws_bytes, void* stream_,
+                                                  float* stage_ms_host) {
+  if (!stage_ms_host) return MOTE_ERR_NULL;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  for (int i = 0; i < MOTE_N_STAGES; ++i) stage_ms_host[i] = 0.0f;
+  for (int i = 0; i <= MOTE_N_STAGES; ++i) MOTE_CUDA_OK(cudaEventCreate(&g_timer.ev[i]));
+  g_timer.active = true;
+  mote_status_t st = mote_moe_forward(L, x, residual, T, out, nullptr, ws, ws_bytes, stream);
+  g_timer.active = false;
+  if (st == MOTE_OK && T > 0) {
+    if (cudaStreamSynchronize(stream) != cudaSuccess) st = MOTE_ERR_CUDA;
+    for (int i = 0; st == MOTE_OK && i < MOTE_N_STAGES; ++i)
+      if (cudaEventElapsedTime(&stage_ms_host[i], g_timer.ev[i], g_timer.ev[i + 1]) != cudaSuccess) st = MOTE_ERR_CUDA;
+  }
+  for (int i = 0; i <= MOTE_N_STAGES; ++i) cudaEventDestroy(g_timer.ev[i]);
+  return st;
 }

@@ -6,7 +6,7 @@ import torch
 
 from oracle import mote_oracle as O
 from workloads import synth
-from tests.parity_utils import bf16_bits, bf16_tensor, check_forward, check_packed_layer
+from parity_utils import bf16_bits, bf16_tensor, check_forward, check_packed_layer
 
 pytestmark = pytest.mark.gpu
 

@@ -6,7 +6,7 @@ import torch
 
 from oracle import mote_oracle as O
 from workloads import synth
-from tests.parity_utils import bf16_bits, bf16_tensor
+from parity_utils import bf16_bits, bf16_tensor
 
 pytestmark = pytest.mark.gpu
 
