@@ -15,7 +15,9 @@ constexpr int kDispatchThreads = 1024;
 __global__ void __launch_bounds__(kDispatchThreads) dispatch_kernel(const int32_t* __restrict__ idx, int P, int E,
                                                                     int32_t* __restrict__ offsets,
                                                                     int32_t* __restrict__ perm,
-                                                                    int32_t* __restrict__ inv) {
+                                                                    int32_t* __restrict__ inv,
+                                                                    int4* __restrict__ tiles_routed,
+                                                                    int4* __restrict__ tiles_shared, int T) {
   __shared__ int s_count[MOTE_MAX_EXPERTS];
   __shared__ int s_running[MOTE_MAX_EXPERTS];
   __shared__ int s_warp[32][MOTE_MAX_EXPERTS];
@@ -37,6 +39,21 @@ __global__ void __launch_bounds__(kDispatchThreads) dispatch_kernel(const int32_
       run += s_count[e];
     }
     offsets[E] = run;
+  }
+  // row-tile tables of the tensor-core GEMMs: [0] = {count}, [1+i] = {expert, first row, rows}
+  if (tid == 32 && tiles_routed) {
+    int n = 0, run = 0;
+    for (int e = 0; e < E; ++e) {
+      const int cnt = s_count[e];
+      for (int r = 0; r < cnt; r += 128) tiles_routed[1 + n++] = make_int4(e, run + r, min(128, cnt - r), 0);
+      run += cnt;
+    }
+    tiles_routed[0] = make_int4(n, 0, 0, 0);
+  }
+  if (tiles_shared) {
+    const int n = (T + 127) / 128;
+    for (int i = tid; i < n; i += kDispatchThreads) tiles_shared[1 + i] = make_int4(0, i * 128, min(128, T - i * 128), 0);
+    if (tid == 0) tiles_shared[0] = make_int4(n, 0, 0, 0);
   }
   __syncthreads();
 
@@ -68,8 +85,10 @@ __global__ void __launch_bounds__(kDispatchThreads) dispatch_kernel(const int32_
 }
 
 mote_status_t launch_dispatch(const int32_t* idx, int64_t P, int E, int32_t* offsets, int32_t* perm,
-                              int32_t* inv, cudaStream_t stream) {
-  dispatch_kernel<<<1, kDispatchThreads, 0, stream>>>(idx, (int)P, E, offsets, perm, inv);
+                              int32_t* inv, int4* tiles_routed, int4* tiles_shared, int64_t T,
+                              cudaStream_t stream) {
+  dispatch_kernel<<<1, kDispatchThreads, 0, stream>>>(idx, (int)P, E, offsets, perm, inv, tiles_routed,
+                                                      tiles_shared, (int)T);
   ++g_launch_count;
   MOTE_LAUNCH_OK();
   return MOTE_OK;

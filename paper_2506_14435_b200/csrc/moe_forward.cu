@@ -25,7 +25,7 @@ static inline void stage_mark(int i, cudaStream_t stream) {
 
 struct Plan {
   size_t status, topk_idx, topk_w, offsets, perm, inv;
-  size_t qx, beta_x, rowsum_x, h, qh, beta_h, rowsum_h, y, hs, s;
+  size_t qx, beta_x, rowsum_x, h, qh, beta_h, rowsum_h, y, hs, s, tiles_routed, tiles_shared;
   size_t total;
 };
 
@@ -50,6 +50,8 @@ static Plan make_plan(int d, int f, int E, int k, int64_t T) {
   p.y = take(P * size_t(d) * 4);
   p.hs = take(size_t(T) * f * 2);
   p.s = take(size_t(T) * d * 4);
+  p.tiles_routed = take((1 + P / 128 + E) * 16);
+  p.tiles_shared = take((1 + (size_t(T) + 127) / 128) * 16);
   p.total = off;
   return p;
 }
@@ -173,17 +175,29 @@ extern "C" mote_status_t mote_moe_forward(const mote_layer_t* L, const void* x, 
   void* hs = base + pl.hs;
   auto* s = reinterpret_cast<float*>(base + pl.s);
 
-  const int path = (L->path == MOTE_PATH_AUTO) ? MOTE_PATH_SIMT : L->path;
-  if (path != MOTE_PATH_SIMT) return MOTE_ERR_SHAPE;     // other paths are wired in below as they land
-  const int interleave = 0;
+  auto* tiles_routed = reinterpret_cast<int4*>(base + pl.tiles_routed);
+  auto* tiles_shared = reinterpret_cast<int4*>(base + pl.tiles_shared);
+  auto* status = reinterpret_cast<uint32_t*>(base + pl.status);
+  const int max_mtiles_routed = (int)(P / 128 + E);
+  const int max_mtiles_shared = (int)((T + 127) / 128);
+
+  const bool tensor_ok = (d % 128 == 0) && (f % 128 == 0);
+  int path = L->path;
+  if (path == MOTE_PATH_AUTO) path = tensor_ok ? MOTE_PATH_TENSOR : MOTE_PATH_SIMT;
+  if (path == MOTE_PATH_STREAM) return MOTE_ERR_SHAPE;   // not available yet
+  if (path == MOTE_PATH_TENSOR && !tensor_ok) return MOTE_ERR_SHAPE;
+  const bool tensor = (path == MOTE_PATH_TENSOR);
+  const int interleave = tensor ? 1 : 0;
 
   mote_status_t st;
+  MOTE_CUDA_OK(cudaMemsetAsync(status, 0, 4, stream));
   stage_mark(0, stream);
   // S1 router, S2 dispatch
   st = launch_route_topk(x, T, d, L->Wr, L->router_bias, E, k, L->norm_topk, topk_idx, topk_w, nullptr, stream);
   if (st) return st;
   stage_mark(1, stream);
-  st = launch_dispatch(topk_idx, P, E, offsets, perm, inv, stream);
+  st = launch_dispatch(topk_idx, P, E, offsets, perm, inv, tensor ? tiles_routed : nullptr,
+                       tensor ? tiles_shared : nullptr, T, stream);
   if (st) return st;
   stage_mark(2, stream);
   // S3 Q_a(x), written once per selected expert into the expert-sorted rows
@@ -198,7 +212,8 @@ extern "C" mote_status_t mote_moe_forward(const mote_layer_t* L, const void* x, 
   g1.qa = qx; g1.beta = beta_x; g1.offsets = offsets; g1.w0 = L->gate_packed; g1.w1 = L->up_packed;
   g1.alpha0 = L->alpha_gate; g1.alpha1 = L->alpha_up; g1.E = E; g1.N = f; g1.K = d; g1.P = P;
   g1.h_bf16 = h; g1.acc0_tap = taps ? taps->acc_gate : nullptr; g1.acc1_tap = taps ? taps->acc_up : nullptr;
-  st = launch_ternary_gateup_simt(g1, stream);
+  st = tensor ? launch_ternary_umma(g1, true, tiles_routed, max_mtiles_routed, rowsum_x, status, stream)
+              : launch_ternary_gateup_simt(g1, stream);
   if (st) return st;
   stage_mark(4, stream);
   // S5 Q_a(h)
@@ -212,14 +227,19 @@ extern "C" mote_status_t mote_moe_forward(const mote_layer_t* L, const void* x, 
   TernaryGemmArgs g2{};
   g2.qa = qh; g2.beta = beta_h; g2.offsets = offsets; g2.w0 = L->down_packed; g2.alpha0 = L->alpha_down;
   g2.E = E; g2.N = d; g2.K = f; g2.P = P; g2.y = y; g2.acc0_tap = taps ? taps->acc_down : nullptr;
-  st = launch_ternary_down_simt(g2, stream);
+  st = tensor ? launch_ternary_umma(g2, false, tiles_routed, max_mtiles_routed, rowsum_h, status, stream)
+              : launch_ternary_down_simt(g2, stream);
   if (st) return st;
   stage_mark(6, stream);
   // S7 shared expert
-  st = launch_shared_gateup_simt(x, L->sh_gate, L->sh_up, T, d, f, hs, stream);
+  st = tensor ? launch_shared_umma(x, L->sh_gate, L->sh_up, true, T, d, f, hs, tiles_shared, max_mtiles_shared,
+                                   status, stream)
+              : launch_shared_gateup_simt(x, L->sh_gate, L->sh_up, T, d, f, hs, stream);
   if (st) return st;
   stage_mark(7, stream);
-  st = launch_shared_down_simt(hs, L->sh_down, T, d, f, s, stream);
+  st = tensor ? launch_shared_umma(hs, L->sh_down, nullptr, false, T, f, d, s, tiles_shared, max_mtiles_shared,
+                                   status, stream)
+              : launch_shared_down_simt(hs, L->sh_down, T, d, f, s, stream);
   if (st) return st;
   stage_mark(8, stream);
   // S8 combine

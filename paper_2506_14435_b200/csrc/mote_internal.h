@@ -29,8 +29,12 @@ mote_status_t launch_route_topk(const void* x, int64_t T, int d, const float* Wr
                                 cudaStream_t stream);
 
 // Stable grouping of the T*k pairs by expert: offsets[E+1], perm[P] (pair -> row), inv[P] (row -> pair).
+// Optionally also writes the 128-row tile tables of the tensor-core GEMMs ([0] = {count},
+// [1+i] = {expert, first row, rows}); tiles_routed needs 1 + P/128 + E entries, tiles_shared
+// 1 + ceil(T/128).
 mote_status_t launch_dispatch(const int32_t* idx, int64_t P, int E, int32_t* offsets, int32_t* perm,
-                              int32_t* inv, cudaStream_t stream);
+                              int32_t* inv, int4* tiles_routed, int4* tiles_shared, int64_t T,
+                              cudaStream_t stream);
 
 // CUDA-core (dp4a) grouped ternary GEMMs.  qa rows are in expert-sorted order, canonical k order.
 struct TernaryGemmArgs {
@@ -51,6 +55,14 @@ struct TernaryGemmArgs {
 };
 mote_status_t launch_ternary_gateup_simt(const TernaryGemmArgs& a, cudaStream_t stream);
 mote_status_t launch_ternary_down_simt(const TernaryGemmArgs& a, cudaStream_t stream);
+
+// Tensor-core (tcgen05) versions.  qa must be stored k-interleaved (see quant_act.cu); needs
+// K % 128 == 0 and N % 128 == 0.
+mote_status_t launch_ternary_umma(const TernaryGemmArgs& a, bool gateup, const int4* tiles, int max_mtiles,
+                                  const int32_t* rowsum, uint32_t* status, cudaStream_t stream);
+mote_status_t launch_shared_umma(const void* act, const void* w0, const void* w1, bool gateup, int64_t T, int K,
+                                 int N, void* out, const int4* tiles, int max_mtiles, uint32_t* status,
+                                 cudaStream_t stream);
 
 // CUDA-core bf16 GEMMs of the shared expert.
 mote_status_t launch_shared_gateup_simt(const void* x, const void* Wg, const void* Wu, int64_t T, int d,

@@ -1,0 +1,495 @@
+// Tensor-core expert GEMMs for sm_100a: tcgen05.mma with TMEM accumulators, operands staged in
+// shared memory by TMA, warp-specialised persistent CTAs (one per SM).
+//
+//   T_GATEUP  routed gate/up (Eq. 6): int8 tokens x 2-bit weights -> int32; epilogue applies
+//             the dequantisation scales, SiLU and the gate*up product, writes h as bf16
+//   T_DOWN    routed down (Eq. 5): int8 Q_a(h) x 2-bit weights -> int32 -> y fp32
+//   B_GATEUP  shared expert gate/up (Eq. 2): bf16 x bf16 -> fp32 -> h_shared bf16
+//   B_DOWN    shared expert down -> s fp32
+//
+// Tile: 128 token rows (UMMA M, one TMEM lane per row) x BN weight rows (UMMA N = 256, or 128 for
+// a down projection whose width is not a multiple of 256); K advances 128 bytes of the token
+// operand per pipeline stage (128 int8 or 64 bf16), four K=32-byte MMAs per stage.
+//
+// Ternary weights travel as 2-bit codes all the way into shared memory (TMA box of 32 bytes per
+// weight row and stage) and are expanded there to int8 by four unpacker warps, directly into the
+// 128-byte-swizzled operand layout the MMA reads.  The stored code is code+1 in {0,1,2}, so the
+// expansion is a shift and a mask ((w >> 2i) & 0x03030303); the weights enter the MMA as
+// UNSIGNED int8 and the epilogue subtracts the token's row sum (sum_k q_k) to recover
+// sum_k q_k * code_k exactly.  The shift/mask yields the 16 codes of a word in the order
+// 0,4,8,12,1,5,...; the token operand is stored in the same order by the activation quantizer,
+// and an integer dot product does not depend on the order of its terms.
+//
+// Warp roles (384 threads): 0 TMA producer of the token operand (and of bf16 weights),
+// 1 TMA producer of packed weights, 2 MMA issuer + TMEM owner, 4-7 unpackers, 8-11 epilogue.
+// Two accumulator buffers of 256 TMEM columns let the epilogue of one tile overlap the MMAs of
+// the next.  Every mbarrier wait is bounded; on expiry the CTA raises a status word and leaves.
+#include <cuda.h>
+
+#include <algorithm>
+#include <mutex>
+
+#include "mote_common.cuh"
+#include "mote_internal.h"
+#include "ptx_sm100.cuh"
+
+namespace mote {
+
+using namespace ptx;
+
+enum { MODE_T_GATEUP = 0, MODE_T_DOWN = 1, MODE_B_GATEUP = 2, MODE_B_DOWN = 3 };
+
+constexpr int kBM = 128;
+constexpr int kStageA = kBM * 128;             // 16 KB: 128 rows x 128 B
+constexpr int kStageB = 256 * 128;             // 32 KB: up to 256 rows x 128 B
+constexpr int kStageP = 256 * 32;              // 8 KB: up to 256 rows x 32 B of packed codes
+constexpr int kStagesTernary = 3, kStagesP = 4, kStagesBf16 = 4;
+constexpr int kThreads = 384;
+constexpr int kTmemCols = 512;
+
+struct UmmaArgs {
+  const int4* tiles;        // [0] = {n_mtiles,0,0,0}; [1+i] = {expert, row0, rows, 0}
+  int n_ntiles;             // tiles along the output columns
+  int k_steps;              // pipeline stages along K (128 bytes of the token operand each)
+  int bn;                   // weight rows per tile (UMMA N)
+  int n_out;                // output row length (f for gate/up, d for down)
+  int b_rows_per_expert;    // rows of the weight tensor map per expert (0: shared expert)
+  const float* beta;        // [rows]   (ternary modes)
+  const int32_t* rowsum;    // [rows]
+  const float* alpha0;      // [E]
+  const float* alpha1;      // [E] (gate/up: alpha_up)
+  void* out;                // bf16 [rows, n_out] (gate/up) or fp32 [rows, n_out] (down)
+  int32_t* tap0;            // optional int32 [rows, n_out]
+  int32_t* tap1;
+  uint32_t* status;
+};
+
+struct __align__(8) PipeBarriers {
+  uint64_t full_a[4], empty[4], full_u[4], full_p[4], empty_p[4], tmem_full[2], tmem_empty[2];
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+template <int MODE>
+struct ModeTraits {
+  static constexpr bool kTernary = (MODE == MODE_T_GATEUP || MODE == MODE_T_DOWN);
+  static constexpr bool kGateUp = (MODE == MODE_T_GATEUP || MODE == MODE_B_GATEUP);
+  static constexpr int kStages = kTernary ? kStagesTernary : kStagesBf16;
+  static constexpr size_t kSmem =
+      1024 + size_t(kStages) * (kStageA + kStageB) + (kTernary ? size_t(kStagesP) * kStageP : 0) + sizeof(PipeBarriers);
+};
+
+__device__ __forceinline__ void decode_item(const UmmaArgs& a, int item, int n_mtiles, int4& tile, int& n_tile) {
+  const int m_tile = item % n_mtiles;
+  n_tile = item / n_mtiles;
+  tile = a.tiles[1 + m_tile];
+}
+
+// ------------------------------------------------------------------------------------------------
+template <int MODE>
+__global__ void __launch_bounds__(kThreads, 1)
+umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b0,
+                 const __grid_constant__ CUtensorMap tm_b1, const UmmaArgs a) {
+  using TR = ModeTraits<MODE>;
+  constexpr int S = TR::kStages;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+  const uint32_t sA = smem_base;
+  const uint32_t sB = sA + S * kStageA;
+  const uint32_t sP = sB + S * kStageB;
+  uint8_t* genB = smem_gen + S * kStageA;
+  uint8_t* genP = genB + S * kStageB;
+  PipeBarriers* bars = reinterpret_cast<PipeBarriers*>(genP + (TR::kTernary ? kStagesP * kStageP : 0));
+  volatile int* abort_flag = &bars->abort_flag;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n_mtiles = a.tiles[0].x;
+  const int n_items = n_mtiles * a.n_ntiles;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < 4; ++s) {
+      mbar_init(smem_u32(&bars->full_a[s]), 1);
+      mbar_init(smem_u32(&bars->empty[s]), 1);
+      mbar_init(smem_u32(&bars->full_u[s]), 4);
+      mbar_init(smem_u32(&bars->full_p[s]), 1);
+      mbar_init(smem_u32(&bars->empty_p[s]), 4);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(smem_u32(&bars->tmem_full[b]), 1);
+      mbar_init(smem_u32(&bars->tmem_empty[b]), 4);
+    }
+    bars->abort_flag = 0;
+    fence_barrier_init();
+    prefetch_tensormap(&tm_a);
+    prefetch_tensormap(&tm_b0);
+    prefetch_tensormap(&tm_b1);
+  }
+  if (warp == 2) {
+    tmem_alloc(smem_u32(&bars->tmem_base), kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = bars->tmem_base;
+
+  if (warp == 0) {
+    // ---------------------------------------------------------------- token-operand producer
+    if (lane == 0) {
+      uint32_t stage = 0, phase = 0;
+      bool ok = true;
+      for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x) {
+        int4 tile; int n_tile;
+        decode_item(a, item, n_mtiles, tile, n_tile);
+        const int b_row = (a.b_rows_per_expert ? tile.x * a.b_rows_per_expert : 0) + n_tile * (TR::kGateUp ? a.bn / 2 : a.bn);
+        for (int ks = 0; ks < a.k_steps; ++ks) {
+          if (!(ok = mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1, abort_flag))) break;
+          const uint32_t bar = smem_u32(&bars->full_a[stage]);
+          if (TR::kTernary) {
+            mbar_expect_tx(bar, kStageA);
+            tma_load_2d(sA + stage * kStageA, &tm_a, ks * 128, tile.y, bar);
+          } else {
+            mbar_expect_tx(bar, kStageA + a.bn * 128);
+            tma_load_2d(sA + stage * kStageA, &tm_a, ks * 64, tile.y, bar);
+            if (TR::kGateUp) {
+              tma_load_2d(sB + stage * kStageB, &tm_b0, ks * 64, b_row, bar);
+              tma_load_2d(sB + stage * kStageB + 128 * 128, &tm_b1, ks * 64, b_row, bar);
+            } else {
+              tma_load_2d(sB + stage * kStageB, &tm_b0, ks * 64, b_row, bar);
+              if (a.bn == 256) tma_load_2d(sB + stage * kStageB + 128 * 128, &tm_b0, ks * 64, b_row + 128, bar);
+            }
+          }
+          if (++stage == S) { stage = 0; phase ^= 1; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------------------------------------------------------- packed-weight producer
+    if (TR::kTernary && lane == 0) {
+      uint32_t stage = 0, phase = 0;
+      bool ok = true;
+      for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x) {
+        int4 tile; int n_tile;
+        decode_item(a, item, n_mtiles, tile, n_tile);
+        const int b_row = tile.x * a.b_rows_per_expert + n_tile * (TR::kGateUp ? a.bn / 2 : a.bn);
+        for (int ks = 0; ks < a.k_steps; ++ks) {
+          if (!(ok = mbar_wait(smem_u32(&bars->empty_p[stage]), phase ^ 1, abort_flag))) break;
+          const uint32_t bar = smem_u32(&bars->full_p[stage]);
+          mbar_expect_tx(bar, a.bn * 32);
+          const uint32_t dst = sP + stage * kStageP;
+          if (TR::kGateUp) {
+            tma_load_2d(dst, &tm_b0, ks * 32, b_row, bar);
+            tma_load_2d(dst + 128 * 32, &tm_b1, ks * 32, b_row, bar);
+          } else {
+            tma_load_2d(dst, &tm_b0, ks * 32, b_row, bar);
+            if (a.bn == 256) tma_load_2d(dst + 128 * 32, &tm_b0, ks * 32, b_row + 128, bar);
+          }
+          if (++stage == kStagesP) { stage = 0; phase ^= 1; }
+        }
+      }
+    }
+  } else if (warp == 2) {
+    // ---------------------------------------------------------------- MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc = TR::kTernary ? make_idesc(2, 1, 0, kBM, (uint32_t)a.bn)     // s32 += s8 * u8
+                                          : make_idesc(1, 1, 1, kBM, (uint32_t)a.bn);    // f32 += bf16 * bf16
+      uint32_t stage = 0, phase = 0;
+      int local = 0;
+      bool ok = true;
+      for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x, ++local) {
+        const int buf = local & 1;
+        const uint32_t use = (uint32_t)(local >> 1);
+        if (!(ok = mbar_wait(smem_u32(&bars->tmem_empty[buf]), (use & 1) ^ 1, abort_flag))) break;
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + buf * 256;
+        for (int ks = 0; ks < a.k_steps; ++ks) {
+          if (!(ok = mbar_wait(smem_u32(&bars->full_a[stage]), phase, abort_flag))) break;
+          if (TR::kTernary)
+            if (!(ok = mbar_wait(smem_u32(&bars->full_u[stage]), phase, abort_flag))) break;
+          tc_fence_after();
+          const uint64_t da = smem_desc_sw128(sA + stage * kStageA);
+          const uint64_t db = smem_desc_sw128(sB + stage * kStageB);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const uint32_t acc = (ks > 0 || j > 0) ? 1u : 0u;
+            if (TR::kTernary) mma_i8(d_tmem, da + 2 * j, db + 2 * j, idesc, acc);
+            else mma_f16(d_tmem, da + 2 * j, db + 2 * j, idesc, acc);
+          }
+          mma_commit(smem_u32(&bars->empty[stage]));
+          if (++stage == S) { stage = 0; phase ^= 1; }
+        }
+        if (ok) mma_commit(smem_u32(&bars->tmem_full[buf]));
+      }
+    }
+  } else if (warp >= 4 && warp < 8) {
+    // ---------------------------------------------------------------- 2-bit -> int8 unpackers
+    if (TR::kTernary) {
+      const int tid = threadIdx.x - 128;
+      uint32_t stage = 0, phase = 0, pstage = 0, pphase = 0;
+      bool ok = true;
+      const int chunks_per_thread = a.bn / 64;       // bn*2 chunks of 16 packed bytes over 128 threads
+      for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x) {
+        for (int ks = 0; ks < a.k_steps; ++ks) {
+          ok = mbar_wait(smem_u32(&bars->full_p[pstage]), pphase, abort_flag) &&
+               mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1, abort_flag);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          const uint8_t* src = genP + pstage * kStageP;
+          uint8_t* dst = genB + stage * kStageB;
+          for (int i = 0; i < chunks_per_thread; ++i) {
+            const int c = i * 128 + tid;
+            const int r = c >> 1, half = c & 1;
+            const uint4 w = *reinterpret_cast<const uint4*>(src + c * 16);
+            const uint32_t pw[4] = {w.x, w.y, w.z, w.w};
+            uint8_t* row = dst + (r >> 3) * 1024 + (r & 7) * 128;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              uint4 o;
+              o.x = pw[j] & 0x03030303u;
+              o.y = (pw[j] >> 2) & 0x03030303u;
+              o.z = (pw[j] >> 4) & 0x03030303u;
+              o.w = (pw[j] >> 6) & 0x03030303u;
+              *reinterpret_cast<uint4*>(row + (((half * 4 + j) ^ (r & 7)) << 4)) = o;
+            }
+          }
+          fence_proxy_async_smem();                  // generic-proxy writes -> visible to the MMA
+          __syncwarp();
+          if (lane == 0) {
+            mbar_arrive(smem_u32(&bars->full_u[stage]));
+            mbar_arrive(smem_u32(&bars->empty_p[pstage]));
+          }
+          if (++stage == S) { stage = 0; phase ^= 1; }
+          if (++pstage == kStagesP) { pstage = 0; pphase ^= 1; }
+        }
+      }
+    }
+  } else if (warp >= 8) {
+    // ---------------------------------------------------------------- epilogue
+    const int q = warp & 3;                          // TMEM lane quarter this warp may read
+    const int r_in_tile = q * 32 + lane;
+    int local = 0;
+    bool ok = true;
+    for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x, ++local) {
+      int4 tile; int n_tile;
+      decode_item(a, item, n_mtiles, tile, n_tile);
+      const int buf = local & 1;
+      const uint32_t use = (uint32_t)(local >> 1);
+      ok = mbar_wait(smem_u32(&bars->tmem_full[buf]), use & 1, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      const bool row_ok = r_in_tile < tile.z;
+      const int64_t row = int64_t(tile.y) + r_in_tile;
+      const uint32_t t_row = tmem_base + (uint32_t(q * 32) << 16) + buf * 256;
+      float c0 = 0.f, c1 = 0.f;
+      int rs = 0;
+      if (TR::kTernary && row_ok) {
+        const float beta = a.beta[row];
+        rs = a.rowsum[row];
+        c0 = dequant_scale(a.alpha0[tile.x], beta);
+        if (TR::kGateUp) c1 = dequant_scale(a.alpha1[tile.x], beta);
+      }
+      if (TR::kGateUp) {
+        const int col0 = n_tile * 128;
+#pragma unroll 1
+        for (int c = 0; c < 128; c += 32) {
+          uint32_t rg[32], ru[32];
+          tmem_ld_32x32b_x32(t_row + c, rg);
+          tmem_ld_32x32b_x32(t_row + 128 + c, ru);
+          tmem_wait_ld();
+          if (row_ok) {
+            uint32_t packed[16];
+#pragma unroll
+            for (int j = 0; j < 32; j += 2) {
+              float h0, h1;
+              if (TR::kTernary) {
+                h0 = glu_h((int)rg[j] - rs, (int)ru[j] - rs, c0, c1);
+                h1 = glu_h((int)rg[j + 1] - rs, (int)ru[j + 1] - rs, c0, c1);
+              } else {
+                const float g0 = __uint_as_float(rg[j]), g1 = __uint_as_float(rg[j + 1]);
+                h0 = __uint_as_float(ru[j]) * (g0 / (1.0f + __expf(-g0)));
+                h1 = __uint_as_float(ru[j + 1]) * (g1 / (1.0f + __expf(-g1)));
+              }
+              packed[j / 2] = f32_to_bf16_bits(h0) | (f32_to_bf16_bits(h1) << 16);
+            }
+            uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<uint16_t*>(a.out) + row * a.n_out + col0 + c);
+#pragma unroll
+            for (int v = 0; v < 4; ++v) dst[v] = make_uint4(packed[4 * v], packed[4 * v + 1], packed[4 * v + 2], packed[4 * v + 3]);
+            if (TR::kTernary && a.tap0) {
+              int4* t0 = reinterpret_cast<int4*>(a.tap0 + row * a.n_out + col0 + c);
+              int4* t1 = reinterpret_cast<int4*>(a.tap1 + row * a.n_out + col0 + c);
+#pragma unroll
+              for (int v = 0; v < 8; ++v) {
+                t0[v] = make_int4((int)rg[4 * v] - rs, (int)rg[4 * v + 1] - rs, (int)rg[4 * v + 2] - rs, (int)rg[4 * v + 3] - rs);
+                t1[v] = make_int4((int)ru[4 * v] - rs, (int)ru[4 * v + 1] - rs, (int)ru[4 * v + 2] - rs, (int)ru[4 * v + 3] - rs);
+              }
+            }
+          }
+        }
+      } else {
+        const int col0 = n_tile * a.bn;
+#pragma unroll 1
+        for (int c = 0; c < a.bn; c += 32) {
+          uint32_t ra[32];
+          tmem_ld_32x32b_x32(t_row + c, ra);
+          tmem_wait_ld();
+          if (row_ok) {
+            float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(a.out) + row * a.n_out + col0 + c);
+#pragma unroll
+            for (int v = 0; v < 8; ++v) {
+              float4 o;
+              if (TR::kTernary) {
+                o.x = __fmul_rn(__int2float_rn((int)ra[4 * v] - rs), c0);
+                o.y = __fmul_rn(__int2float_rn((int)ra[4 * v + 1] - rs), c0);
+                o.z = __fmul_rn(__int2float_rn((int)ra[4 * v + 2] - rs), c0);
+                o.w = __fmul_rn(__int2float_rn((int)ra[4 * v + 3] - rs), c0);
+              } else {
+                o = make_float4(__uint_as_float(ra[4 * v]), __uint_as_float(ra[4 * v + 1]),
+                                __uint_as_float(ra[4 * v + 2]), __uint_as_float(ra[4 * v + 3]));
+              }
+              dst[v] = o;
+            }
+            if (TR::kTernary && a.tap0) {
+              int4* t0 = reinterpret_cast<int4*>(a.tap0 + row * a.n_out + col0 + c);
+#pragma unroll
+              for (int v = 0; v < 8; ++v)
+                t0[v] = make_int4((int)ra[4 * v] - rs, (int)ra[4 * v + 1] - rs, (int)ra[4 * v + 2] - rs, (int)ra[4 * v + 3] - rs);
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&bars->tmem_empty[buf]));
+    }
+  }
+
+  // ------------------------------------------------------------------ teardown
+  if (*abort_flag) {
+    // give copies and MMAs still in flight time to land before shared memory and TMEM go away
+    const uint64_t t0 = globaltimer_ns();
+    while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 2) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+  if (threadIdx.x == 0 && *abort_flag) atomicExch(a.status, 1u);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Host side: tensor maps and launches
+// ------------------------------------------------------------------------------------------------
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  });
+  return fn;
+}
+
+// 2-D row-major tensor [rows, cols] of elem_bytes-wide elements, box [box_rows, box_cols].
+static bool make_map_2d(CUtensorMap* m, const void* base, CUtensorMapDataType dt, int elem_bytes, uint64_t rows,
+                        uint64_t cols, uint32_t box_rows, uint32_t box_cols, CUtensorMapSwizzle sw) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {cols * (uint64_t)elem_bytes};
+  cuuint32_t box[2] = {box_cols, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(m, dt, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int MODE>
+static mote_status_t launch_umma(const CUtensorMap& ta, const CUtensorMap& tb0, const CUtensorMap& tb1,
+                                 const UmmaArgs& a, int max_items, cudaStream_t stream) {
+  using TR = ModeTraits<MODE>;
+  static bool attr_set = false;
+  if (!attr_set) {
+    MOTE_CUDA_OK(cudaFuncSetAttribute(umma_gemm_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TR::kSmem));
+    attr_set = true;
+  }
+  int dev = 0, sms = 148;
+  MOTE_CUDA_OK(cudaGetDevice(&dev));
+  MOTE_CUDA_OK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+  const int grid = std::max(1, std::min(sms, max_items));
+  umma_gemm_kernel<MODE><<<grid, kThreads, TR::kSmem, stream>>>(ta, tb0, tb1, a);
+  ++g_launch_count;
+  MOTE_LAUNCH_OK();
+  return MOTE_OK;
+}
+
+mote_status_t launch_ternary_umma(const TernaryGemmArgs& g, bool gateup, const int4* tiles, int max_mtiles,
+                                  const int32_t* rowsum, uint32_t* status, cudaStream_t stream) {
+  if (g.P == 0) return MOTE_OK;
+  CUtensorMap ta, tb0, tb1;
+  const int bn = gateup ? 256 : ((g.N % 256 == 0) ? 256 : 128);
+  if (!make_map_2d(&ta, g.qa, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)g.P, (uint64_t)g.K, 128, 128,
+                   CU_TENSOR_MAP_SWIZZLE_128B))
+    return MOTE_ERR_CUDA;
+  if (!make_map_2d(&tb0, g.w0, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)g.E * g.N, (uint64_t)g.K / 4, 128, 32,
+                   CU_TENSOR_MAP_SWIZZLE_NONE))
+    return MOTE_ERR_CUDA;
+  if (!make_map_2d(&tb1, gateup ? g.w1 : g.w0, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)g.E * g.N,
+                   (uint64_t)g.K / 4, 128, 32, CU_TENSOR_MAP_SWIZZLE_NONE))
+    return MOTE_ERR_CUDA;
+  UmmaArgs a{};
+  a.tiles = tiles;
+  a.n_ntiles = gateup ? g.N / 128 : g.N / bn;
+  a.k_steps = g.K / 128;
+  a.bn = bn;
+  a.n_out = g.N;
+  a.b_rows_per_expert = g.N;
+  a.beta = g.beta; a.rowsum = rowsum; a.alpha0 = g.alpha0; a.alpha1 = g.alpha1;
+  a.out = gateup ? g.h_bf16 : static_cast<void*>(g.y);
+  a.tap0 = g.acc0_tap; a.tap1 = g.acc1_tap;
+  a.status = status;
+  const int max_items = max_mtiles * a.n_ntiles;
+  return gateup ? launch_umma<MODE_T_GATEUP>(ta, tb0, tb1, a, max_items, stream)
+                : launch_umma<MODE_T_DOWN>(ta, tb0, tb1, a, max_items, stream);
+}
+
+mote_status_t launch_shared_umma(const void* act, const void* w0, const void* w1, bool gateup, int64_t T, int K,
+                                 int N, void* out, const int4* tiles, int max_mtiles, uint32_t* status,
+                                 cudaStream_t stream) {
+  if (T == 0) return MOTE_OK;
+  CUtensorMap ta, tb0, tb1;
+  const int bn = gateup ? 256 : ((N % 256 == 0) ? 256 : 128);
+  if (!make_map_2d(&ta, act, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)T, (uint64_t)K, 128, 64,
+                   CU_TENSOR_MAP_SWIZZLE_128B))
+    return MOTE_ERR_CUDA;
+  if (!make_map_2d(&tb0, w0, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)N, (uint64_t)K, 128, 64,
+                   CU_TENSOR_MAP_SWIZZLE_128B))
+    return MOTE_ERR_CUDA;
+  if (!make_map_2d(&tb1, gateup ? w1 : w0, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)N, (uint64_t)K, 128, 64,
+                   CU_TENSOR_MAP_SWIZZLE_128B))
+    return MOTE_ERR_CUDA;
+  UmmaArgs a{};
+  a.tiles = tiles;
+  a.n_ntiles = gateup ? N / 128 : N / bn;
+  a.k_steps = K / 64;
+  a.bn = bn;
+  a.n_out = N;
+  a.b_rows_per_expert = 0;
+  a.out = out;
+  a.status = status;
+  const int max_items = max_mtiles * a.n_ntiles;
+  return gateup ? launch_umma<MODE_B_GATEUP>(ta, tb0, tb1, a, max_items, stream)
+                : launch_umma<MODE_B_DOWN>(ta, tb0, tb1, a, max_items, stream);
+}
+
+}  // namespace mote

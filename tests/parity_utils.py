@@ -43,6 +43,7 @@ def check_forward(mote, layer_gpu, layer_or: dict, x_bits: np.ndarray, residual_
     out_buf = res if out_alias_residual else None
     out = mote.mote_moe_forward(layer_gpu, x, residual=res, out=out_buf, taps=taps)
     torch.cuda.synchronize()
+    assert mote.lib.mote_device_status(layer_gpu._ws.data_ptr(), None) == 0, "a device-side wait timed out"
     g = {n: t.cpu() for n, t in taps.items()}
     g_idx = g["topk_idx"].numpy()
 

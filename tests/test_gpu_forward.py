@@ -10,7 +10,8 @@ from parity_utils import bf16_bits, bf16_tensor, check_forward, check_packed_lay
 
 pytestmark = pytest.mark.gpu
 
-PATHS = {"simt": 1}
+SIMT, TENSOR = 1, 2
+BOTH = [pytest.param(SIMT, id="simt"), pytest.param(TENSOR, id="tensor")]
 
 
 @pytest.fixture(scope="module")
@@ -26,35 +27,42 @@ def _setup(mote, wl, path=1):
     return master, layer_or, layer_gpu
 
 
-def test_c1_full_parity(mote):
+@pytest.mark.parametrize("path", BOTH)
+def test_c1_full_parity(mote, path):
     wl = synth.WORKLOADS["c1"]
-    master, layer_or, layer_gpu = _setup(mote, wl)
+    master, layer_or, layer_gpu = _setup(mote, wl, path)
     check_packed_layer(layer_gpu, layer_or)
     rep = check_forward(mote, layer_gpu, layer_or, synth.tokens(wl))
     assert rep["rel_fro"] < 5e-3
 
 
-@pytest.mark.parametrize("d,f,E,k,T,kw", [
-    (16, 32, 3, 2, 5, {}),
-    (48, 80, 2, 1, 1, {}),
-    (64, 112, 5, 5, 33, {}),                       # k = E
-    (256, 512, 4, 2, 300, dict(outlier_frac=0.02)),
-    (128, 256, 8, 2, 77, dict(bias="zipf")),
-    (128, 384, 4, 1, 130, dict(norm_topk=0)),
+@pytest.mark.parametrize("d,f,E,k,T,kw,path", [
+    (16, 32, 3, 2, 5, {}, SIMT),
+    (48, 80, 2, 1, 1, {}, SIMT),
+    (64, 112, 5, 5, 33, {}, SIMT),                       # k = E
+    (256, 512, 4, 2, 300, dict(outlier_frac=0.02), SIMT),
+    (128, 256, 8, 2, 77, dict(bias="zipf"), SIMT),
+    (128, 384, 4, 1, 130, dict(norm_topk=0), SIMT),
+    (128, 128, 2, 1, 1, {}, TENSOR),                      # one row, one k-step
+    (256, 512, 4, 2, 300, dict(outlier_frac=0.02), TENSOR),   # ragged tails in every expert
+    (128, 256, 8, 2, 77, dict(bias="zipf"), TENSOR),
+    (128, 384, 4, 1, 130, dict(norm_topk=0), TENSOR),     # down projection with 128-wide tiles
+    (384, 640, 3, 3, 515, {}, TENSOR),                    # k = E, several row tiles per expert
 ])
-def test_small_shapes(mote, d, f, E, k, T, kw):
+def test_small_shapes(mote, d, f, E, k, T, kw, path):
     wl = synth.custom("small", d, f, E, k, T, 2000 + d + f + T, **kw)
-    master, layer_or, layer_gpu = _setup(mote, wl)
+    master, layer_or, layer_gpu = _setup(mote, wl, path)
     check_packed_layer(layer_gpu, layer_or)
     check_forward(mote, layer_gpu, layer_or, synth.tokens(wl))
 
 
-def test_idle_and_overloaded_experts_residual_and_aliasing(mote):
+@pytest.mark.parametrize("path", BOTH)
+def test_idle_and_overloaded_experts_residual_and_aliasing(mote, path):
     wl = synth.custom("skew", 128, 256, 4, 2, 97, 3001)
     master = synth.master_layer(wl)
     master["router_bias"] = np.array([50.0, -50.0, 40.0, -60.0], np.float32)   # experts 1 and 3 idle
     layer_or = O.build_layer(master)
-    layer_gpu = mote.MoteLayer.from_master(master, path=1)
+    layer_gpu = mote.MoteLayer.from_master(master, path=path)
     x = synth.tokens(wl)
     res = synth.tokens(wl, stream=1)
     rep = check_forward(mote, layer_gpu, layer_or, x, residual_bits=res)
@@ -63,9 +71,10 @@ def test_idle_and_overloaded_experts_residual_and_aliasing(mote):
     assert torch.equal(rep["out"], rep2["out"])
 
 
-def test_run_to_run_determinism_and_token_permutation(mote):
+@pytest.mark.parametrize("path", BOTH)
+def test_run_to_run_determinism_and_token_permutation(mote, path):
     wl = synth.custom("det", 256, 512, 4, 2, 200, 3002)
-    master, layer_or, layer_gpu = _setup(mote, wl)
+    master, layer_or, layer_gpu = _setup(mote, wl, path)
     x = bf16_tensor(synth.tokens(wl))
     a = mote.mote_moe_forward(layer_gpu, x).clone()
     b = mote.mote_moe_forward(layer_gpu, x).clone()
@@ -83,9 +92,11 @@ def test_zero_tokens_is_a_noop(mote):
     assert out.shape == (0, wl.d)
 
 
+@pytest.mark.parametrize("path", BOTH)
 @pytest.mark.parametrize("T", synth.C3_BATCHES)
-def test_c3_decode_batches(mote, T, c3_layers):
+def test_c3_decode_batches(mote, T, path, c3_layers):
     wl, layer_or, layer_gpu = c3_layers
+    layer_gpu.path = path
     rep = check_forward(mote, layer_gpu, layer_or, synth.tokens(wl, T=T))
     assert rep["rel_fro"] < 5e-3
 
