@@ -212,7 +212,10 @@ extern "C" mote_status_t mote_moe_forward(const mote_layer_t* L, const void* x, 
   g1.qa = qx; g1.beta = beta_x; g1.offsets = offsets; g1.w0 = L->gate_packed; g1.w1 = L->up_packed;
   g1.alpha0 = L->alpha_gate; g1.alpha1 = L->alpha_up; g1.E = E; g1.N = f; g1.K = d; g1.P = P;
   g1.h_bf16 = h; g1.acc0_tap = taps ? taps->acc_gate : nullptr; g1.acc1_tap = taps ? taps->acc_up : nullptr;
-  st = tensor ? launch_ternary_umma(g1, true, tiles_routed, max_mtiles_routed, rowsum_x, status, stream)
+  if (tensor)   // beta_h (atomicMax target) and rowsum_h (atomicAdd target) are adjacent
+    MOTE_CUDA_OK(cudaMemsetAsync(beta_h, 0, (pl.rowsum_h - pl.beta_h) + size_t(P) * 4, stream));
+  st = tensor ? launch_ternary_umma(g1, true, tiles_routed, max_mtiles_routed, rowsum_x,
+                                    reinterpret_cast<uint32_t*>(beta_h), status, stream)
               : launch_ternary_gateup_simt(g1, stream);
   if (st) return st;
   stage_mark(4, stream);
@@ -220,14 +223,15 @@ extern "C" mote_status_t mote_moe_forward(const mote_layer_t* L, const void* x, 
   QuantActArgs qb{};
   qb.x = h; qb.T = P; qb.d = f; qb.ldx = f; qb.q = qh; qb.beta = beta_h; qb.rowsum = rowsum_h;
   qb.perm = nullptr; qb.k = 1; qb.interleave = interleave;
-  st = launch_quant_act(qb, false, stream);
+  st = tensor ? launch_quant_rows_known_beta(h, P, f, qh, beta_h, rowsum_h, interleave, stream)
+              : launch_quant_act(qb, false, stream);
   if (st) return st;
   stage_mark(5, stream);
   // S6 down
   TernaryGemmArgs g2{};
   g2.qa = qh; g2.beta = beta_h; g2.offsets = offsets; g2.w0 = L->down_packed; g2.alpha0 = L->alpha_down;
   g2.E = E; g2.N = d; g2.K = f; g2.P = P; g2.y = y; g2.acc0_tap = taps ? taps->acc_down : nullptr;
-  st = tensor ? launch_ternary_umma(g2, false, tiles_routed, max_mtiles_routed, rowsum_h, status, stream)
+  st = tensor ? launch_ternary_umma(g2, false, tiles_routed, max_mtiles_routed, rowsum_h, nullptr, status, stream)
               : launch_ternary_down_simt(g2, stream);
   if (st) return st;
   stage_mark(6, stream);

@@ -44,11 +44,12 @@ __device__ __forceinline__ uint32_t f32_to_bf16_bits(float x) {
 // ---------------------------------------------------------------------------------------------
 // Eq. 8: q = clamp(rint((127*x)/beta), -128, 127); 127*x is exact for a bf16 x.
 // ---------------------------------------------------------------------------------------------
+// |127*x/beta| <= 127 whenever beta >= |x|, so the nearest-even integer can be read from the
+// low bits of (v + 1.5*2^23); the clamp is applied to that integer.
 __device__ __forceinline__ int quant_one(float x, float beta) {
-  float t = __fmul_rn(127.0f, x);
-  float r = rintf(__fdiv_rn(t, beta));
-  r = fminf(fmaxf(r, -128.0f), 127.0f);
-  return __float2int_rn(r);
+  const float v = __fdiv_rn(__fmul_rn(127.0f, x), beta);
+  const int q = __float_as_int(__fadd_rn(fminf(fmaxf(v, -1024.0f), 1024.0f), 12582912.0f)) - 0x4B400000;
+  return min(max(q, -128), 127);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -58,10 +59,22 @@ __device__ __forceinline__ int quant_one(float x, float beta) {
 //   p = c6;  p = p*r + c_i  (i = 5..0), c_i = fl32(ln2^i / i!)
 //   E = p * 2^n;   silu = g / (1 + E)
 // ---------------------------------------------------------------------------------------------
+//
+// Two exact shortcuts keep the instruction count down without changing a single bit:
+//   * rint(t) for |t| <= 125 is (t + 1.5*2^23) - 1.5*2^23 in round-to-nearest-even, and the
+//     low bits of (t + 1.5*2^23) hold the integer n, so p * 2^n is an integer add of n << 23
+//     to the bits of p (p in [0.70, 1.42], n in [-125, 125]: no overflow, no subnormals);
+//   * fl32(acc) for |acc| < 2^22 is bits(acc + 0x4B400000) - 1.5*2^23 (an integer add and an
+//     exact float subtract) instead of a conversion instruction.
+constexpr float kMagic = 12582912.0f;          // 1.5 * 2^23 = bits 0x4B400000
+
+__device__ __forceinline__ float i2f_small(int a) { return __fsub_rn(__int_as_float(a + 0x4B400000), kMagic); }
+
 __device__ __forceinline__ float exp_neg_pinned(float g) {
   float t = __fmul_rn(-g, 1.4426950408889634f);
   t = fminf(fmaxf(t, -125.0f), 125.0f);
-  float n = rintf(t);
+  const float tm = __fadd_rn(t, kMagic);
+  float n = __fsub_rn(tm, kMagic);
   float r = __fsub_rn(t, n);
   float p = 1.5403530393381609e-4f;                       // ln2^6/720
   p = __fadd_rn(__fmul_rn(p, r), 1.3333558146428443e-3f); // ln2^5/120
@@ -70,8 +83,7 @@ __device__ __forceinline__ float exp_neg_pinned(float g) {
   p = __fadd_rn(__fmul_rn(p, r), 2.4022650695910071e-1f); // ln2^2/2
   p = __fadd_rn(__fmul_rn(p, r), 6.9314718055994531e-1f); // ln2
   p = __fadd_rn(__fmul_rn(p, r), 1.0f);
-  float scale = __int_as_float((__float2int_rn(n) + 127) << 23);
-  return __fmul_rn(p, scale);
+  return __int_as_float(__float_as_int(p) + (__float_as_int(tm) << 23));
 }
 
 __device__ __forceinline__ float silu_pinned(float g) {
@@ -80,9 +92,16 @@ __device__ __forceinline__ float silu_pinned(float g) {
 
 // h = bf16_rn(u * silu(g)),  g = fl32(acc_g) * c_g,  u = fl32(acc_u) * c_u
 __device__ __forceinline__ float glu_h(int acc_g, int acc_u, float c_g, float c_u) {
-  float g = __fmul_rn(__int2float_rn(acc_g), c_g);
-  float u = __fmul_rn(__int2float_rn(acc_u), c_u);
+  float g = __fmul_rn(i2f_small(acc_g), c_g);
+  float u = __fmul_rn(i2f_small(acc_u), c_u);
   return __fmul_rn(u, silu_pinned(g));
+}
+
+// two floats -> packed bf16x2 (round to nearest even), lo in the low half
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  uint32_t d;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+  return d;
 }
 
 // scale of one ternary linear output row: alpha * (beta / 127)

@@ -58,8 +58,15 @@ mote_status_t launch_ternary_down_simt(const TernaryGemmArgs& a, cudaStream_t st
 
 // Tensor-core (tcgen05) versions.  qa must be stored k-interleaved (see quant_act.cu); needs
 // K % 128 == 0 and N % 128 == 0.
+// beta_out_bits (gate/up only, may be null): per row, atomicMax of the bits of |h| (must be zeroed).
 mote_status_t launch_ternary_umma(const TernaryGemmArgs& a, bool gateup, const int4* tiles, int max_mtiles,
-                                  const int32_t* rowsum, uint32_t* status, cudaStream_t stream);
+                                  const int32_t* rowsum, uint32_t* beta_out_bits, uint32_t* status,
+                                  cudaStream_t stream);
+
+// Q_a(h) for rows whose absmax is already known: beta_bits holds max |h| per row (raw bits);
+// writes q (k-interleaved if asked), the clamped beta in place, and accumulates rowsum (zeroed).
+mote_status_t launch_quant_rows_known_beta(const void* h_bf16, int64_t rows, int n, int8_t* q, float* beta,
+                                           int32_t* rowsum, int interleave, cudaStream_t stream);
 mote_status_t launch_shared_umma(const void* act, const void* w0, const void* w1, bool gateup, int64_t T, int K,
                                  int N, void* out, const int4* tiles, int max_mtiles, uint32_t* status,
                                  cudaStream_t stream);

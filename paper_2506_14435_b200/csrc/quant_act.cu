@@ -119,6 +119,64 @@ __global__ void __launch_bounds__(256) quant_act_kernel(QuantActArgs a) {
   }
 }
 
+// Q_a(h) when the row maxima are already known (the gate/up GEMM epilogue accumulates them with
+// atomicMax): a pure streaming pass, one unit of 16 elements per thread and iteration.
+__global__ void __launch_bounds__(256) quant_rows_known_beta_kernel(const uint4* __restrict__ h, int64_t n_units_total,
+                                                                    int units_per_row, uint4* __restrict__ q,
+                                                                    float* beta, int32_t* __restrict__ rowsum,
+                                                                    int interleave) {
+  const int lane = threadIdx.x & 31;
+  const int64_t stride = int64_t(gridDim.x) * blockDim.x;
+  const int64_t first = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
+  for (int64_t base = first - lane; base < n_units_total; base += stride) {
+    const int64_t u = base + lane;
+    const bool ok = u < n_units_total;
+    int row = -1, sum = 0;
+    if (ok) {
+      row = (int)(u / units_per_row);
+      const float b = fmaxf(beta[row], kEpsScale);
+      const uint4 r0 = h[u * 2], r1 = h[u * 2 + 1];
+      const uint32_t w[8] = {r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w};
+      int qv[16];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        qv[2 * j] = quant_one(bf16_lo(w[j]), b);
+        qv[2 * j + 1] = quant_one(bf16_hi(w[j]), b);
+      }
+      uint32_t o[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        if (interleave)
+          o[i] = (qv[i] & 0xFF) | ((qv[4 + i] & 0xFF) << 8) | ((qv[8 + i] & 0xFF) << 16) | ((qv[12 + i] & 0xFF) << 24);
+        else
+          o[i] = (qv[4 * i] & 0xFF) | ((qv[4 * i + 1] & 0xFF) << 8) | ((qv[4 * i + 2] & 0xFF) << 16) |
+                 ((qv[4 * i + 3] & 0xFF) << 24);
+      }
+#pragma unroll
+      for (int j = 0; j < 16; ++j) sum += qv[j];
+      q[u] = make_uint4(o[0], o[1], o[2], o[3]);
+      if (u - int64_t(row) * units_per_row == 0) beta[row] = b;   // publish the clamped scale
+    }
+    // one atomic per (warp, row)
+    const unsigned peers = __match_any_sync(0xffffffffu, row);
+    const int total = __reduce_add_sync(peers, sum);
+    if (ok && lane == (__ffs(peers) - 1)) atomicAdd(rowsum + row, total);
+  }
+}
+
+mote_status_t launch_quant_rows_known_beta(const void* h_bf16, int64_t rows, int n, int8_t* q, float* beta,
+                                           int32_t* rowsum, int interleave, cudaStream_t stream) {
+  if (rows == 0) return MOTE_OK;
+  const int units_per_row = n / 16;
+  const int64_t total = rows * units_per_row;
+  const unsigned blocks = (unsigned)std::min<int64_t>((total + 255) / 256, 148 * 8);
+  quant_rows_known_beta_kernel<<<blocks, 256, 0, stream>>>(static_cast<const uint4*>(h_bf16), total, units_per_row,
+                                                           reinterpret_cast<uint4*>(q), beta, rowsum, interleave);
+  ++g_launch_count;
+  MOTE_LAUNCH_OK();
+  return MOTE_OK;
+}
+
 mote_status_t launch_quant_act(const QuantActArgs& a, bool scatter, cudaStream_t stream) {
   if (a.T == 0) return MOTE_OK;
   const int n_units = a.d / 16;

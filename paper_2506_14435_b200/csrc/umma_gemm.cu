@@ -20,8 +20,10 @@
 // 0,4,8,12,1,5,...; the token operand is stored in the same order by the activation quantizer,
 // and an integer dot product does not depend on the order of its terms.
 //
-// Warp roles (384 threads): 0 TMA producer of the token operand (and of bf16 weights),
-// 1 TMA producer of packed weights, 2 MMA issuer + TMEM owner, 4-7 unpackers, 8-11 epilogue.
+// Warp roles (640 threads): 0 TMA producer of the token operand (and of bf16 weights),
+// 1 TMA producer of packed weights, 2 MMA issuer + TMEM owner, 4-11 two groups of unpackers
+// that take alternate pipeline stages, 12-19 epilogue (two warps per TMEM lane quarter, each
+// owning half of the tile's columns).
 // Two accumulator buffers of 256 TMEM columns let the epilogue of one tile overlap the MMAs of
 // the next.  Every mbarrier wait is bounded; on expiry the CTA raises a status word and leaves.
 #include <cuda.h>
@@ -44,7 +46,7 @@ constexpr int kStageA = kBM * 128;             // 16 KB: 128 rows x 128 B
 constexpr int kStageB = 256 * 128;             // 32 KB: up to 256 rows x 128 B
 constexpr int kStageP = 256 * 32;              // 8 KB: up to 256 rows x 32 B of packed codes
 constexpr int kStagesTernary = 3, kStagesP = 4, kStagesBf16 = 4;
-constexpr int kThreads = 384;
+constexpr int kThreads = 640;
 constexpr int kTmemCols = 512;
 
 struct UmmaArgs {
@@ -61,6 +63,7 @@ struct UmmaArgs {
   void* out;                // bf16 [rows, n_out] (gate/up) or fp32 [rows, n_out] (down)
   int32_t* tap0;            // optional int32 [rows, n_out]
   int32_t* tap1;
+  uint32_t* beta_out_bits;  // gate/up of the routed experts: running max |h| per row (atomicMax on the bits)
   uint32_t* status;
 };
 
@@ -117,7 +120,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(smem_u32(&bars->tmem_full[b]), 1);
-      mbar_init(smem_u32(&bars->tmem_empty[b]), 4);
+      mbar_init(smem_u32(&bars->tmem_empty[b]), 8);
     }
     bars->abort_flag = 0;
     fence_barrier_init();
@@ -222,51 +225,56 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
         if (ok) mma_commit(smem_u32(&bars->tmem_full[buf]));
       }
     }
-  } else if (warp >= 4 && warp < 8) {
+  } else if (warp >= 4 && warp < 12) {
     // ---------------------------------------------------------------- 2-bit -> int8 unpackers
+    // group 0 (warps 4-7) expands the even pipeline steps, group 1 (warps 8-11) the odd ones
     if (TR::kTernary) {
-      const int tid = threadIdx.x - 128;
-      uint32_t stage = 0, phase = 0, pstage = 0, pphase = 0;
+      const int group = (warp - 4) >> 2;
+      const int tid = (threadIdx.x - 128) & 127;
+      uint32_t stage = 0, phase = 0, pstage = 0, pphase = 0, step = 0;
       bool ok = true;
       const int chunks_per_thread = a.bn / 64;       // bn*2 chunks of 16 packed bytes over 128 threads
       for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x) {
-        for (int ks = 0; ks < a.k_steps; ++ks) {
-          ok = mbar_wait(smem_u32(&bars->full_p[pstage]), pphase, abort_flag) &&
-               mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1, abort_flag);
-          ok = __all_sync(0xffffffffu, ok);
-          if (!ok) break;
-          const uint8_t* src = genP + pstage * kStageP;
-          uint8_t* dst = genB + stage * kStageB;
-          for (int i = 0; i < chunks_per_thread; ++i) {
-            const int c = i * 128 + tid;
-            const int r = c >> 1, half = c & 1;
-            const uint4 w = *reinterpret_cast<const uint4*>(src + c * 16);
-            const uint32_t pw[4] = {w.x, w.y, w.z, w.w};
-            uint8_t* row = dst + (r >> 3) * 1024 + (r & 7) * 128;
+        for (int ks = 0; ks < a.k_steps; ++ks, ++step) {
+          if ((step & 1u) == (uint32_t)group) {
+            ok = mbar_wait(smem_u32(&bars->full_p[pstage]), pphase, abort_flag) &&
+                 mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1, abort_flag);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            const uint8_t* src = genP + pstage * kStageP;
+            uint8_t* dst = genB + stage * kStageB;
+            for (int i = 0; i < chunks_per_thread; ++i) {
+              const int c = i * 128 + tid;
+              const int r = c >> 1, half = c & 1;
+              const uint4 w = *reinterpret_cast<const uint4*>(src + c * 16);
+              const uint32_t pw[4] = {w.x, w.y, w.z, w.w};
+              uint8_t* row = dst + (r >> 3) * 1024 + (r & 7) * 128;
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              uint4 o;
-              o.x = pw[j] & 0x03030303u;
-              o.y = (pw[j] >> 2) & 0x03030303u;
-              o.z = (pw[j] >> 4) & 0x03030303u;
-              o.w = (pw[j] >> 6) & 0x03030303u;
-              *reinterpret_cast<uint4*>(row + (((half * 4 + j) ^ (r & 7)) << 4)) = o;
+              for (int j = 0; j < 4; ++j) {
+                uint4 o;
+                o.x = pw[j] & 0x03030303u;
+                o.y = (pw[j] >> 2) & 0x03030303u;
+                o.z = (pw[j] >> 4) & 0x03030303u;
+                o.w = (pw[j] >> 6) & 0x03030303u;
+                *reinterpret_cast<uint4*>(row + (((half * 4 + j) ^ (r & 7)) << 4)) = o;
+              }
             }
-          }
-          fence_proxy_async_smem();                  // generic-proxy writes -> visible to the MMA
-          __syncwarp();
-          if (lane == 0) {
-            mbar_arrive(smem_u32(&bars->full_u[stage]));
-            mbar_arrive(smem_u32(&bars->empty_p[pstage]));
+            fence_proxy_async_smem();                // generic-proxy writes -> visible to the MMA
+            __syncwarp();
+            if (lane == 0) {
+              mbar_arrive(smem_u32(&bars->full_u[stage]));
+              mbar_arrive(smem_u32(&bars->empty_p[pstage]));
+            }
           }
           if (++stage == S) { stage = 0; phase ^= 1; }
           if (++pstage == kStagesP) { pstage = 0; pphase ^= 1; }
         }
       }
     }
-  } else if (warp >= 8) {
+  } else if (warp >= 12) {
     // ---------------------------------------------------------------- epilogue
     const int q = warp & 3;                          // TMEM lane quarter this warp may read
+    const int chalf = (warp - 12) >> 2;              // which half of the tile's columns
     const int r_in_tile = q * 32 + lane;
     int local = 0;
     bool ok = true;
@@ -285,23 +293,24 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
       float c0 = 0.f, c1 = 0.f;
       int rs = 0;
       if (TR::kTernary && row_ok) {
-        const float beta = a.beta[row];
+        const float beta = fmaxf(a.beta[row], kEpsScale);
         rs = a.rowsum[row];
         c0 = dequant_scale(a.alpha0[tile.x], beta);
         if (TR::kGateUp) c1 = dequant_scale(a.alpha1[tile.x], beta);
       }
       if (TR::kGateUp) {
         const int col0 = n_tile * 128;
+        uint32_t hmax = 0u;                          // max |h| of this thread's elements, as bf16 bits << 16
 #pragma unroll 1
-        for (int c = 0; c < 128; c += 32) {
-          uint32_t rg[32], ru[32];
-          tmem_ld_32x32b_x32(t_row + c, rg);
-          tmem_ld_32x32b_x32(t_row + 128 + c, ru);
+        for (int c = chalf * 64; c < chalf * 64 + 64; c += 16) {
+          uint32_t rg[16], ru[16];
+          tmem_ld_32x32b_x16(t_row + c, rg);
+          tmem_ld_32x32b_x16(t_row + 128 + c, ru);
           tmem_wait_ld();
           if (row_ok) {
-            uint32_t packed[16];
+            uint32_t packed[8];
 #pragma unroll
-            for (int j = 0; j < 32; j += 2) {
+            for (int j = 0; j < 16; j += 2) {
               float h0, h1;
               if (TR::kTernary) {
                 h0 = glu_h((int)rg[j] - rs, (int)ru[j] - rs, c0, c1);
@@ -311,39 +320,44 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
                 h0 = __uint_as_float(ru[j]) * (g0 / (1.0f + __expf(-g0)));
                 h1 = __uint_as_float(ru[j + 1]) * (g1 / (1.0f + __expf(-g1)));
               }
-              packed[j / 2] = f32_to_bf16_bits(h0) | (f32_to_bf16_bits(h1) << 16);
+              const uint32_t pk = pack_bf16x2(h0, h1);
+              packed[j / 2] = pk;
+              if (TR::kTernary) hmax = max(hmax, max((pk << 16) & 0x7FFFFFFFu, pk & 0x7FFF0000u));
             }
             uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<uint16_t*>(a.out) + row * a.n_out + col0 + c);
-#pragma unroll
-            for (int v = 0; v < 4; ++v) dst[v] = make_uint4(packed[4 * v], packed[4 * v + 1], packed[4 * v + 2], packed[4 * v + 3]);
+            dst[0] = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+            dst[1] = make_uint4(packed[4], packed[5], packed[6], packed[7]);
             if (TR::kTernary && a.tap0) {
               int4* t0 = reinterpret_cast<int4*>(a.tap0 + row * a.n_out + col0 + c);
               int4* t1 = reinterpret_cast<int4*>(a.tap1 + row * a.n_out + col0 + c);
 #pragma unroll
-              for (int v = 0; v < 8; ++v) {
+              for (int v = 0; v < 4; ++v) {
                 t0[v] = make_int4((int)rg[4 * v] - rs, (int)rg[4 * v + 1] - rs, (int)rg[4 * v + 2] - rs, (int)rg[4 * v + 3] - rs);
                 t1[v] = make_int4((int)ru[4 * v] - rs, (int)ru[4 * v + 1] - rs, (int)ru[4 * v + 2] - rs, (int)ru[4 * v + 3] - rs);
               }
             }
           }
         }
+        // bits of non-negative floats order like unsigned integers
+        if (TR::kTernary && row_ok && a.beta_out_bits && hmax) atomicMax(a.beta_out_bits + row, hmax);
       } else {
         const int col0 = n_tile * a.bn;
+        const int cbeg = chalf * (a.bn / 2), cend = cbeg + a.bn / 2;
 #pragma unroll 1
-        for (int c = 0; c < a.bn; c += 32) {
-          uint32_t ra[32];
-          tmem_ld_32x32b_x32(t_row + c, ra);
+        for (int c = cbeg; c < cend; c += 16) {
+          uint32_t ra[16];
+          tmem_ld_32x32b_x16(t_row + c, ra);
           tmem_wait_ld();
           if (row_ok) {
             float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(a.out) + row * a.n_out + col0 + c);
 #pragma unroll
-            for (int v = 0; v < 8; ++v) {
+            for (int v = 0; v < 4; ++v) {
               float4 o;
               if (TR::kTernary) {
-                o.x = __fmul_rn(__int2float_rn((int)ra[4 * v] - rs), c0);
-                o.y = __fmul_rn(__int2float_rn((int)ra[4 * v + 1] - rs), c0);
-                o.z = __fmul_rn(__int2float_rn((int)ra[4 * v + 2] - rs), c0);
-                o.w = __fmul_rn(__int2float_rn((int)ra[4 * v + 3] - rs), c0);
+                o.x = __fmul_rn(i2f_small((int)ra[4 * v] - rs), c0);
+                o.y = __fmul_rn(i2f_small((int)ra[4 * v + 1] - rs), c0);
+                o.z = __fmul_rn(i2f_small((int)ra[4 * v + 2] - rs), c0);
+                o.w = __fmul_rn(i2f_small((int)ra[4 * v + 3] - rs), c0);
               } else {
                 o = make_float4(__uint_as_float(ra[4 * v]), __uint_as_float(ra[4 * v + 1]),
                                 __uint_as_float(ra[4 * v + 2]), __uint_as_float(ra[4 * v + 3]));
@@ -353,7 +367,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
             if (TR::kTernary && a.tap0) {
               int4* t0 = reinterpret_cast<int4*>(a.tap0 + row * a.n_out + col0 + c);
 #pragma unroll
-              for (int v = 0; v < 8; ++v)
+              for (int v = 0; v < 4; ++v)
                 t0[v] = make_int4((int)ra[4 * v] - rs, (int)ra[4 * v + 1] - rs, (int)ra[4 * v + 2] - rs, (int)ra[4 * v + 3] - rs);
             }
           }
@@ -434,7 +448,8 @@ static mote_status_t launch_umma(const CUtensorMap& ta, const CUtensorMap& tb0, 
 }
 
 mote_status_t launch_ternary_umma(const TernaryGemmArgs& g, bool gateup, const int4* tiles, int max_mtiles,
-                                  const int32_t* rowsum, uint32_t* status, cudaStream_t stream) {
+                                  const int32_t* rowsum, uint32_t* beta_out_bits, uint32_t* status,
+                                  cudaStream_t stream) {
   if (g.P == 0) return MOTE_OK;
   CUtensorMap ta, tb0, tb1;
   const int bn = gateup ? 256 : ((g.N % 256 == 0) ? 256 : 128);
@@ -457,6 +472,7 @@ mote_status_t launch_ternary_umma(const TernaryGemmArgs& g, bool gateup, const i
   a.beta = g.beta; a.rowsum = rowsum; a.alpha0 = g.alpha0; a.alpha1 = g.alpha1;
   a.out = gateup ? g.h_bf16 : static_cast<void*>(g.y);
   a.tap0 = g.acc0_tap; a.tap1 = g.acc1_tap;
+  a.beta_out_bits = gateup ? beta_out_bits : nullptr;
   a.status = status;
   const int max_items = max_mtiles * a.n_ntiles;
   return gateup ? launch_umma<MODE_T_GATEUP>(ta, tb0, tb1, a, max_items, stream)
