@@ -37,7 +37,8 @@ typedef enum {
   MOTE_ERR_WORKSPACE = 4,      /* workspace missing or too small                                */
   MOTE_ERR_DTYPE = 5,          /* unknown dtype code                                            */
   MOTE_ERR_CUDA = 6,           /* a CUDA call or launch failed                                  */
-  MOTE_ERR_DEVICE_TIMEOUT = 7  /* a bounded device-side wait expired (see mote_device_status)   */
+  MOTE_ERR_DEVICE_TIMEOUT = 7, /* a bounded device-side wait expired (see mote_device_status)   */
+  MOTE_ERR_TOO_LARGE = 8       /* more elements than a fixed-capacity entry point accepts       */
 } mote_status_t;
 
 enum { MOTE_DTYPE_F32 = 0, MOTE_DTYPE_BF16 = 1 };
@@ -69,6 +70,36 @@ size_t mote_ternarize_workspace_bytes(void);
 mote_status_t mote_ternarize_pack(const void* W, int w_dtype, int64_t m, int64_t n,
                                   uint8_t* packed, float* alpha,
                                   void* ws, size_t ws_bytes, void* stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * mote_ternarize_pack_static -- mote_ternarize_pack without the `ws` argument.  (The paper has no
+ * counterpart: this is a packaging variant of the same quantizer, same results bit for bit.)
+ *
+ * For callers that cannot hand over device scratch and must not trigger an allocation: code that
+ * runs inside a memory pool whose budget is already fully committed, a plug-in loaded into a host
+ * process that owns every allocation, or a latency-critical loop that cannot afford the
+ * device-wide synchronisation an allocation may imply.
+ * The 256 exponent bins (2 KiB) that the exact sum of |w| needs live in a device array inside the
+ * library image, so every GPU that loads the library carries those 2 KiB until the process ends.
+ * The call itself makes no device allocation of any kind; it issues one memset, three kernels.
+ *
+ *   W, w_dtype, m, n, packed, alpha, stream    exactly as mote_ternarize_pack
+ *
+ * Limits and rules
+ *   - m*n <= MOTE_STATIC_MAX_ELEMENTS (2^31, e.g. a 32768 x 65536 matrix); beyond that the call
+ *     returns MOTE_ERR_TOO_LARGE and launches nothing.  Use mote_ternarize_pack for larger ones.
+ *   - The first call on each device looks up the device address of the array (a host-side query,
+ *     no allocation).  Make that first call outside any stream capture.
+ *   - All calls on one device share the one array, and it keeps what the last call left in it;
+ *     each call clears it on `stream` before use.  Two calls that can overlap on the GPU (issued
+ *     on different streams without an ordering between them, or from two host threads) race on
+ *     the bins and both give undefined alpha and codes: serialise them.
+ * Errors: as mote_ternarize_pack, plus MOTE_ERR_TOO_LARGE; MOTE_ERR_CUDA if the address lookup
+ * fails or the device ordinal is 64 or higher.
+ */
+#define MOTE_STATIC_MAX_ELEMENTS ((int64_t)1 << 31)
+mote_status_t mote_ternarize_pack_static(const void* W, int w_dtype, int64_t m, int64_t n,
+                                         uint8_t* packed, float* alpha, void* stream);
 
 /* ------------------------------------------------------------------------------------------------
  * mote_quant_act -- per-token absmax int8 activation quantizer (Eq. 8, 9, 10).

@@ -42,6 +42,9 @@ lib.mote_ternarize_workspace_bytes.argtypes = []
 lib.mote_ternarize_pack.restype = C.c_int
 lib.mote_ternarize_pack.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p,
                                     C.c_void_p, C.c_size_t, C.c_void_p]
+lib.mote_ternarize_pack_static.restype = C.c_int
+lib.mote_ternarize_pack_static.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p,
+                                           C.c_void_p]
 lib.mote_quant_act.restype = C.c_int
 lib.mote_quant_act.argtypes = [C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p,
                                C.c_void_p, C.c_void_p]
@@ -103,6 +106,21 @@ def mote_ternarize_pack(W: torch.Tensor):
     ws = torch.empty(ws_bytes, dtype=torch.uint8, device=W.device)
     _check(lib.mote_ternarize_pack(_ptr(W), dt, m, n, _ptr(packed), _ptr(alpha), _ptr(ws), ws_bytes, _stream()),
            "mote_ternarize_pack")
+    return packed, alpha
+
+
+def mote_ternarize_pack_static(W: torch.Tensor, packed: torch.Tensor, alpha: torch.Tensor):
+    """mote_ternarize_pack for callers that may not allocate: the caller passes the outputs
+    (packed uint8[m, n/4], alpha float32[1]) and the library uses its built-in 2 KiB of device
+    scratch, so neither this wrapper nor the call behind it allocates device memory.  At most 2^31
+    elements; calls on one device must not overlap (they share the scratch)."""
+    _need_cuda(W, packed, alpha)
+    m, n = W.shape
+    dt = {torch.float32: DTYPE_F32, torch.bfloat16: DTYPE_BF16}[W.dtype]
+    if packed.dtype != torch.uint8 or packed.numel() != m * n // 4 or alpha.dtype != torch.float32:
+        raise ValueError("packed must be uint8[m, n/4] and alpha float32[1]")
+    _check(lib.mote_ternarize_pack_static(_ptr(W), dt, m, n, _ptr(packed), _ptr(alpha), _stream()),
+           "mote_ternarize_pack_static")
     return packed, alpha
 
 

@@ -105,6 +105,7 @@ extern "C" const char* mote_status_string(mote_status_t st) {
     case MOTE_ERR_DTYPE: return "unknown dtype";
     case MOTE_ERR_CUDA: return "CUDA error";
     case MOTE_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+    case MOTE_ERR_TOO_LARGE: return "input larger than this entry point's fixed capacity";
   }
   return "unknown status";
 }

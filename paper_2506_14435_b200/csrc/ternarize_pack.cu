@@ -8,6 +8,9 @@
 //   2. alpha_finalize  one thread adds the bins into a 384-bit integer (exact), rounds it to
 //                      fp64 (nearest even), divides by m*n in fp64 and rounds once to fp32.
 //   3. pack_codes      code = clamp(rint(w / alpha), -1, 1), four codes per byte.
+#include <algorithm>
+#include <mutex>
+
 #include "mote_common.cuh"
 
 namespace mote {
@@ -165,6 +168,71 @@ extern "C" mote_status_t mote_ternarize_pack(const void* W, int w_dtype, int64_t
   const int threads = 256;
   int blocks_a = (int)std::min<int64_t>((n_vec + threads - 1) / threads, 148 * 8);
   int blocks_c = (int)std::min<int64_t>((n_words + threads - 1) / threads, 148 * 16);
+  if (w_dtype == MOTE_DTYPE_BF16)
+    abs_sum_bins_kernel<true><<<blocks_a, threads, 0, stream>>>(W, n_vec, bins);
+  else
+    abs_sum_bins_kernel<false><<<blocks_a, threads, 0, stream>>>(W, n_vec, bins);
+  MOTE_LAUNCH_OK();
+  alpha_finalize_kernel<<<1, 32, 0, stream>>>(bins, (double)total, alpha);
+  MOTE_LAUNCH_OK();
+  if (w_dtype == MOTE_DTYPE_BF16)
+    pack_codes_kernel<true><<<blocks_c, threads, 0, stream>>>(W, n_words, alpha, reinterpret_cast<uint32_t*>(packed));
+  else
+    pack_codes_kernel<false><<<blocks_c, threads, 0, stream>>>(W, n_words, alpha, reinterpret_cast<uint32_t*>(packed));
+  MOTE_LAUNCH_OK();
+  return MOTE_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// mote_ternarize_pack_static: the same quantizer for callers that have no scratch buffer to give.
+// The exponent bins live in a device array that is part of the loaded library image.
+// ---------------------------------------------------------------------------------------------
+namespace mote {
+
+// 256 bins x 8 bytes.  One copy per GPU that loads the library, held until the process exits.
+static __device__ __align__(256) unsigned long long g_static_bins[kBins];
+
+constexpr int kMaxDevices = 64;
+static unsigned long long* g_static_bins_ptr[kMaxDevices];   // device address of g_static_bins, per device
+static std::mutex g_static_bins_mutex;
+
+// In host code `g_static_bins` is only a handle; the kernels need the address the array has on the
+// device that is current.  It is looked up on the first call made on each device.
+static mote_status_t static_bins_address(unsigned long long** out) {
+  int dev = -1;
+  MOTE_CUDA_OK(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return MOTE_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(g_static_bins_mutex);
+  if (!g_static_bins_ptr[dev]) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_bins) != cudaSuccess || !p) return MOTE_ERR_CUDA;
+    g_static_bins_ptr[dev] = static_cast<unsigned long long*>(p);
+  }
+  *out = g_static_bins_ptr[dev];
+  return MOTE_OK;
+}
+
+}  // namespace mote
+
+extern "C" mote_status_t mote_ternarize_pack_static(const void* W, int w_dtype, int64_t m, int64_t n,
+                                                    uint8_t* packed, float* alpha, void* stream_) {
+  using namespace mote;
+  if (!W || !packed || !alpha) return MOTE_ERR_NULL;
+  if (w_dtype != MOTE_DTYPE_F32 && w_dtype != MOTE_DTYPE_BF16) return MOTE_ERR_DTYPE;
+  if (m <= 0 || n <= 0 || (n % 16) != 0) return MOTE_ERR_SHAPE;
+  if (m > MOTE_STATIC_MAX_ELEMENTS / n) return MOTE_ERR_TOO_LARGE;
+  if (!aligned16(W) || !aligned16(packed)) return MOTE_ERR_ALIGN;
+  unsigned long long* bins = nullptr;
+  const mote_status_t st = static_bins_address(&bins);
+  if (st != MOTE_OK) return st;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  const int64_t total = m * n;
+  const int64_t n_vec = total / 4, n_words = total / 16;
+  // the array still holds the previous call's sums
+  MOTE_CUDA_OK(cudaMemsetAsync(bins, 0, kBins * sizeof(unsigned long long), stream));
+  const int threads = 256;
+  const int blocks_a = (int)std::min<int64_t>((n_vec + threads - 1) / threads, 148 * 8);
+  const int blocks_c = (int)std::min<int64_t>((n_words + threads - 1) / threads, 148 * 16);
   if (w_dtype == MOTE_DTYPE_BF16)
     abs_sum_bins_kernel<true><<<blocks_a, threads, 0, stream>>>(W, n_vec, bins);
   else
