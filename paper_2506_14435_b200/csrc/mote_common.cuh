@@ -44,12 +44,45 @@ __device__ __forceinline__ uint32_t f32_to_bf16_bits(float x) {
 // ---------------------------------------------------------------------------------------------
 // Eq. 8: q = clamp(rint((127*x)/beta), -128, 127); 127*x is exact for a bf16 x.
 // ---------------------------------------------------------------------------------------------
+constexpr float kMagic = 12582912.0f;          // 1.5 * 2^23 = bits 0x4B400000
+
 // |127*x/beta| <= 127 whenever beta >= |x|, so the nearest-even integer can be read from the
 // low bits of (v + 1.5*2^23); the clamp is applied to that integer.
 __device__ __forceinline__ int quant_one(float x, float beta) {
   const float v = __fdiv_rn(__fmul_rn(127.0f, x), beta);
-  const int q = __float_as_int(__fadd_rn(fminf(fmaxf(v, -1024.0f), 1024.0f), 12582912.0f)) - 0x4B400000;
+  const int q = __float_as_int(__fadd_rn(fminf(fmaxf(v, -1024.0f), 1024.0f), kMagic)) - 0x4B400000;
   return min(max(q, -128), 127);
+}
+
+// The same integer without a division per element.  Per row: c = fl(127 * fl(1/beta)).  Per
+// element: r = fl(x*c) differs from 127*x/beta by at most 127 * 3 * 2^-24 < 2^-15, and the
+// reference value v = fl(fl(127*x)/beta) by at most 127 * 2^-24 < 2^-17.  If r is farther than
+// 2^-12 from every half-integer, no half-integer lies between r and v or equals either, hence
+// rint(r) == rint(v).  Otherwise (about 5 elements in 10^4) the division is evaluated.
+// Rows whose beta is outside [1e-30, 1e30] (1/beta or x*c could leave the normal range) always
+// take the division.
+struct QaScale {
+  float beta, c;
+  bool fast;
+};
+__device__ __forceinline__ QaScale qa_scale(float beta) {
+  QaScale s;
+  s.beta = beta;
+  s.c = __fmul_rn(127.0f, __fdiv_rn(1.0f, beta));
+  s.fast = beta > 1e-30f && beta < 1e30f;
+  return s;
+}
+// Returns a word whose LOW BYTE is q (two's complement); the upper bytes are unspecified.
+__device__ __forceinline__ uint32_t quant_byte(float x, const QaScale& s) {
+  const float r = __fmul_rn(x, s.c);
+  const float m = __fadd_rn(r, kMagic);
+  const float frac = __fsub_rn(r, __fsub_rn(m, kMagic));
+  if (!(fabsf(frac) < 0.499755859375f) || !s.fast) return (uint32_t)quant_one(x, s.beta);
+  return __float_as_uint(m);
+}
+// low bytes of four words -> one word (a in the lowest byte)
+__device__ __forceinline__ uint32_t pack_low_bytes(uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  return __byte_perm(__byte_perm(a, b, 0x0040), __byte_perm(c, d, 0x0040), 0x5410);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -66,8 +99,6 @@ __device__ __forceinline__ int quant_one(float x, float beta) {
 //     to the bits of p (p in [0.70, 1.42], n in [-125, 125]: no overflow, no subnormals);
 //   * fl32(acc) for |acc| < 2^22 is bits(acc + 0x4B400000) - 1.5*2^23 (an integer add and an
 //     exact float subtract) instead of a conversion instruction.
-constexpr float kMagic = 12582912.0f;          // 1.5 * 2^23 = bits 0x4B400000
-
 __device__ __forceinline__ float i2f_small(int a) { return __fsub_rn(__int_as_float(a + 0x4B400000), kMagic); }
 
 __device__ __forceinline__ float exp_neg_pinned(float g) {
@@ -95,6 +126,30 @@ __device__ __forceinline__ float glu_h(int acc_g, int acc_u, float c_g, float c_
   float g = __fmul_rn(i2f_small(acc_g), c_g);
   float u = __fmul_rn(i2f_small(acc_u), c_u);
   return __fmul_rn(u, silu_pinned(g));
+}
+
+// The same h through the special-function unit, with a flag telling when that is not enough.
+//   E' = ex2.approx(t), t = fl(-g*log2e) as above (relative error <= 2^-22; the polynomial's E is
+//        within 4e-7 of 2^t)                                     -> |E' - E| <= 6.4e-7 * E
+//   den' = fl(1 + E')                                            -> relative distance <= 7.6e-7
+//   s'  = fl(g * rcp.approx(den'))  (rcp: <= 2^-23, product 2^-24) vs s = fl(g / den) -> <= 1.0e-6
+//   h'  = fl(u * s')                                             vs h  -> <= 1.12e-6 < 19 ulp
+// bf16_rn(h') == bf16_rn(h) unless h' lies within 19 fp32 ulps of the midpoint between two bf16
+// values; the flag is raised within 64 ulps of a midpoint (low 16 bits in [0x7FC0, 0x8040]), and
+// for |t| > 64 where the clamp, overflow or gradual underflow could make the two differ more.
+// Flagged elements (about 0.2 %) are recomputed with glu_h.  The caller must also send rows with
+// c_g * c_u <= 1e-12 to glu_h (h' could be subnormal there).
+__device__ __forceinline__ float glu_h_fast(int acc_g, int acc_u, float c_g, float c_u, bool& redo) {
+  const float g = __fmul_rn(i2f_small(acc_g), c_g);
+  const float u = __fmul_rn(i2f_small(acc_u), c_u);
+  const float t = __fmul_rn(-g, 1.4426950408889634f);
+  float e, rc;
+  asm("ex2.approx.f32 %0, %1;" : "=f"(e) : "f"(t));
+  const float den = __fadd_rn(1.0f, e);
+  asm("rcp.approx.f32 %0, %1;" : "=f"(rc) : "f"(den));
+  const float h = __fmul_rn(u, __fmul_rn(g, rc));
+  redo = ((__float_as_uint(h) & 0xFFFFu) - 0x7FC0u) <= 0x80u || !(fabsf(t) <= 64.0f);
+  return h;
 }
 
 // two floats -> packed bf16x2 (round to nearest even), lo in the low half

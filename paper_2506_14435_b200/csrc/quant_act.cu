@@ -64,32 +64,29 @@ __global__ void __launch_bounds__(256) quant_act_kernel(QuantActArgs a) {
     amax = m;
   }
   const float beta = fmaxf(amax, kEpsScale);
+  const QaScale qs = qa_scale(beta);
 
   int local_sum = 0;
   uint4 outw[kUnits];
 #pragma unroll
   for (int u = 0; u < kUnits; ++u) {
-    int q[16];
+    uint32_t q[16];                                // low byte of each word = the int8 code
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
       const uint32_t w[4] = {raw[u][h].x, raw[u][h].y, raw[u][h].z, raw[u][h].w};
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        q[h * 8 + 2 * j] = quant_one(bf16_lo(w[j]), beta);
-        q[h * 8 + 2 * j + 1] = quant_one(bf16_hi(w[j]), beta);
+        q[h * 8 + 2 * j] = quant_byte(bf16_lo(w[j]), qs);
+        q[h * 8 + 2 * j + 1] = quant_byte(bf16_hi(w[j]), qs);
       }
     }
     uint32_t o[4];
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      if (a.interleave)
-        o[i] = (q[i] & 0xFF) | ((q[4 + i] & 0xFF) << 8) | ((q[8 + i] & 0xFF) << 16) | ((q[12 + i] & 0xFF) << 24);
-      else
-        o[i] = (q[4 * i] & 0xFF) | ((q[4 * i + 1] & 0xFF) << 8) | ((q[4 * i + 2] & 0xFF) << 16) |
-               ((q[4 * i + 3] & 0xFF) << 24);
+      o[i] = a.interleave ? pack_low_bytes(q[i], q[4 + i], q[8 + i], q[12 + i])
+                          : pack_low_bytes(q[4 * i], q[4 * i + 1], q[4 * i + 2], q[4 * i + 3]);
+      local_sum = __dp4a((int)o[i], 0x01010101, local_sum);
     }
-#pragma unroll
-    for (int j = 0; j < 16; ++j) local_sum += q[j];
     outw[u] = make_uint4(o[0], o[1], o[2], o[3]);
   }
   local_sum = warp_sum(local_sum);
@@ -135,25 +132,22 @@ __global__ void __launch_bounds__(256) quant_rows_known_beta_kernel(const uint4*
     if (ok) {
       row = (int)(u / units_per_row);
       const float b = fmaxf(beta[row], kEpsScale);
+      const QaScale qs = qa_scale(b);
       const uint4 r0 = h[u * 2], r1 = h[u * 2 + 1];
       const uint32_t w[8] = {r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w};
-      int qv[16];
+      uint32_t qv[16];
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
-        qv[2 * j] = quant_one(bf16_lo(w[j]), b);
-        qv[2 * j + 1] = quant_one(bf16_hi(w[j]), b);
+        qv[2 * j] = quant_byte(bf16_lo(w[j]), qs);
+        qv[2 * j + 1] = quant_byte(bf16_hi(w[j]), qs);
       }
       uint32_t o[4];
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
-        if (interleave)
-          o[i] = (qv[i] & 0xFF) | ((qv[4 + i] & 0xFF) << 8) | ((qv[8 + i] & 0xFF) << 16) | ((qv[12 + i] & 0xFF) << 24);
-        else
-          o[i] = (qv[4 * i] & 0xFF) | ((qv[4 * i + 1] & 0xFF) << 8) | ((qv[4 * i + 2] & 0xFF) << 16) |
-                 ((qv[4 * i + 3] & 0xFF) << 24);
+        o[i] = interleave ? pack_low_bytes(qv[i], qv[4 + i], qv[8 + i], qv[12 + i])
+                          : pack_low_bytes(qv[4 * i], qv[4 * i + 1], qv[4 * i + 2], qv[4 * i + 3]);
+        sum = __dp4a((int)o[i], 0x01010101, sum);
       }
-#pragma unroll
-      for (int j = 0; j < 16; ++j) sum += qv[j];
       q[u] = make_uint4(o[0], o[1], o[2], o[3]);
       if (u - int64_t(row) * units_per_row == 0) beta[row] = b;   // publish the clamped scale
     }

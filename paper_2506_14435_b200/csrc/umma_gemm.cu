@@ -300,7 +300,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
       }
       if (TR::kGateUp) {
         const int col0 = n_tile * 128;
-        uint32_t hmax = 0u;                          // max |h| of this thread's elements, as bf16 bits << 16
+        const bool row_fast = __fmul_rn(c0, c1) > 1e-12f;
+        float hmax = 0.0f;                           // max |h| (before the bf16 rounding, which is monotonic)
 #pragma unroll 1
         for (int c = chalf * 64; c < chalf * 64 + 64; c += 16) {
           uint32_t rg[16], ru[16];
@@ -308,22 +309,33 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
           tmem_ld_32x32b_x16(t_row + 128 + c, ru);
           tmem_wait_ld();
           if (row_ok) {
+            float hv[16];
+            if (TR::kTernary) {
+              uint32_t redo_mask = 0u;
+#pragma unroll
+              for (int j = 0; j < 16; ++j) {
+                bool redo;
+                hv[j] = glu_h_fast((int)rg[j] - rs, (int)ru[j] - rs, c0, c1, redo);
+                if (redo) redo_mask |= 1u << j;
+              }
+              if (!row_fast) redo_mask = 0xFFFFu;
+              if (redo_mask) {
+#pragma unroll
+                for (int j = 0; j < 16; ++j)
+                  if ((redo_mask >> j) & 1u) hv[j] = glu_h((int)rg[j] - rs, (int)ru[j] - rs, c0, c1);
+              }
+#pragma unroll
+              for (int j = 0; j < 16; ++j) hmax = fmaxf(hmax, fabsf(hv[j]));
+            } else {
+#pragma unroll
+              for (int j = 0; j < 16; ++j) {
+                const float g = __uint_as_float(rg[j]);
+                hv[j] = __uint_as_float(ru[j]) * __fdividef(g, 1.0f + __expf(-g));
+              }
+            }
             uint32_t packed[8];
 #pragma unroll
-            for (int j = 0; j < 16; j += 2) {
-              float h0, h1;
-              if (TR::kTernary) {
-                h0 = glu_h((int)rg[j] - rs, (int)ru[j] - rs, c0, c1);
-                h1 = glu_h((int)rg[j + 1] - rs, (int)ru[j + 1] - rs, c0, c1);
-              } else {
-                const float g0 = __uint_as_float(rg[j]), g1 = __uint_as_float(rg[j + 1]);
-                h0 = __uint_as_float(ru[j]) * (g0 / (1.0f + __expf(-g0)));
-                h1 = __uint_as_float(ru[j + 1]) * (g1 / (1.0f + __expf(-g1)));
-              }
-              const uint32_t pk = pack_bf16x2(h0, h1);
-              packed[j / 2] = pk;
-              if (TR::kTernary) hmax = max(hmax, max((pk << 16) & 0x7FFFFFFFu, pk & 0x7FFF0000u));
-            }
+            for (int j = 0; j < 8; ++j) packed[j] = pack_bf16x2(hv[2 * j], hv[2 * j + 1]);
             uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<uint16_t*>(a.out) + row * a.n_out + col0 + c);
             dst[0] = make_uint4(packed[0], packed[1], packed[2], packed[3]);
             dst[1] = make_uint4(packed[4], packed[5], packed[6], packed[7]);
@@ -338,8 +350,11 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
             }
           }
         }
-        // bits of non-negative floats order like unsigned integers
-        if (TR::kTernary && row_ok && a.beta_out_bits && hmax) atomicMax(a.beta_out_bits + row, hmax);
+        // bits of non-negative floats order like unsigned integers; bf16_rn(max) = max(bf16_rn)
+        if (TR::kTernary && row_ok && a.beta_out_bits) {
+          const uint32_t hb = f32_to_bf16_bits(hmax) << 16;
+          if (hb) atomicMax(a.beta_out_bits + row, hb);
+        }
       } else {
         const int col0 = n_tile * a.bn;
         const int cbeg = chalf * (a.bn / 2), cend = cbeg + a.bn / 2;

@@ -44,7 +44,8 @@ def check_forward(mote, layer_gpu, layer_or: dict, x_bits: np.ndarray, residual_
     out = mote.mote_moe_forward(layer_gpu, x, residual=res, out=out_buf, taps=taps)
     torch.cuda.synchronize()
     assert mote.lib.mote_device_status(layer_gpu._ws.data_ptr(), None) == 0, "a device-side wait timed out"
-    g = {n: t.cpu() for n, t in taps.items()}
+    row_taps = ("acc_gate", "acc_up", "h_bf16", "qh", "beta_h", "acc_down", "y")
+    g = {n: t.cpu() for n, t in taps.items() if n not in row_taps and n != "shared_out"}
     g_idx = g["topk_idx"].numpy()
 
     ref = O.moe_forward(layer_or, x_bits, residual_bits, token_subset=token_subset, near_tie_choice=g_idx)
@@ -59,20 +60,24 @@ def check_forward(mote, layer_gpu, layer_or: dict, x_bits: np.ndarray, residual_
     assert np.array_equal(g["perm"].numpy(), ref["perm"])
     assert np.array_equal(g["qx"].numpy(), ref["qx"])
     assert np.array_equal(g["beta_x"].numpy(), ref["beta_x"])
-    rows = ref["rows"]
-    assert np.array_equal(g["acc_gate"].numpy()[rows], ref["acc_gate"])
-    assert np.array_equal(g["acc_up"].numpy()[rows], ref["acc_up"])
-    assert np.array_equal(bf16_bits(g["h_bf16"])[rows], ref["h_bf16"])
-    assert np.array_equal(g["qh"].numpy()[rows], ref["qh"])
-    assert np.array_equal(g["beta_h"].numpy()[rows], ref["beta_h"])
-    assert np.array_equal(g["acc_down"].numpy()[rows], ref["acc_down"])
-    y = g["y"].numpy()[rows].astype(np.float64)
-    assert np.allclose(y, ref["y"], rtol=2e-6, atol=1e-12)
+    # row- and token-indexed taps: only the oracle's rows travel to the host
+    rows_dev = torch.from_numpy(ref["rows"].astype(np.int64)).cuda()
     toks = ref["tokens"]
-    sh = g["shared_out"].numpy()[toks].astype(np.float64)
+    toks_dev = torch.from_numpy(np.asarray(toks, dtype=np.int64)).cuda()
+    for n in row_taps:
+        g[n] = taps[n][rows_dev].cpu()
+    assert np.array_equal(g["acc_gate"].numpy(), ref["acc_gate"])
+    assert np.array_equal(g["acc_up"].numpy(), ref["acc_up"])
+    assert np.array_equal(bf16_bits(g["h_bf16"]), ref["h_bf16"])
+    assert np.array_equal(g["qh"].numpy(), ref["qh"])
+    assert np.array_equal(g["beta_h"].numpy(), ref["beta_h"])
+    assert np.array_equal(g["acc_down"].numpy(), ref["acc_down"])
+    y = g["y"].numpy().astype(np.float64)
+    assert np.allclose(y, ref["y"], rtol=2e-6, atol=1e-12)
+    sh = taps["shared_out"][toks_dev].cpu().numpy().astype(np.float64)
     sh_err = np.linalg.norm(sh - ref["shared_out"]) / max(np.linalg.norm(ref["shared_out"]), 1e-30)
     assert sh_err <= REL_FRO_TOL, sh_err
-    out_f = O.bf16_to_f32(bf16_bits(out))[toks].astype(np.float64)
+    out_f = O.bf16_to_f32(bf16_bits(out[toks_dev])).astype(np.float64)
     err = np.linalg.norm(out_f - ref["out"]) / max(np.linalg.norm(ref["out"]), 1e-30)
     assert err <= REL_FRO_TOL, err
     return dict(rel_fro=err, shared_rel_fro=sh_err, near_ties=int(near.sum()), tokens=len(toks),

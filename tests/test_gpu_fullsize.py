@@ -1,0 +1,50 @@
+"""Parity at the full sizes of the prefill workloads, in the launch configuration bench.py times
+(automatic path selection).  Routing, dispatch and Q_a(x) are compared for every token; the expert
+stages and the output for a token sample the oracle can afford: the tokens owning the first and
+last row of every expert segment, the rows on both sides of every 128- and 256-row tile boundary,
+and a seeded random remainder (tokens are independent of each other, so a sample is a valid check).
+Packed weights and alpha are compared for every matrix."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import mote_oracle as O
+from workloads import synth
+from parity_utils import bf16_tensor, check_forward, check_packed_layer
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def mote():
+    import paper_2506_14435_b200 as m
+    return m
+
+
+def _sampled_parity(mote, wl, n_random, max_boundary_tokens):
+    master = synth.master_layer(wl)
+    layer_or = O.build_layer(master)
+    layer_gpu = mote.MoteLayer.from_master(master)
+    check_packed_layer(layer_gpu, layer_or)
+    x_bits = synth.tokens(wl)
+    r = O.router(x_bits, layer_or["Wr"], layer_or.get("router_bias"), wl.k, wl.norm_topk)
+    offsets, perm, inv = O.dispatch(r["idx"], wl.E)
+    toks = synth.sample_tokens(offsets, inv, wl.k, wl.T, n_random=n_random, seed=wl.seed)
+    if len(toks) > max_boundary_tokens + n_random:
+        rng = np.random.default_rng(wl.seed)
+        toks = np.sort(rng.choice(toks, size=max_boundary_tokens + n_random, replace=False))
+    toks = toks[~r["near_tie"][toks]]          # a near tie may legitimately move a token to another expert
+    rep = check_forward(mote, layer_gpu, layer_or, x_bits, token_subset=toks)
+    assert rep["tokens"] >= min(64, wl.T)
+    return rep
+
+
+def test_c2_full_size_sampled(mote):
+    rep = _sampled_parity(mote, synth.WORKLOADS["c2"], n_random=96, max_boundary_tokens=400)
+    assert rep["rel_fro"] < 5e-3
+
+
+def test_c4_full_size_sampled(mote):
+    rep = _sampled_parity(mote, synth.WORKLOADS["c4"], n_random=64, max_boundary_tokens=200)
+    assert rep["rel_fro"] < 5e-3
+    assert rep["counts"].min() >= 0 and rep["counts"].sum() == 2 * 8192
