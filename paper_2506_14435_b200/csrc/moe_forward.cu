@@ -176,19 +176,73 @@ extern "C" mote_status_t mote_moe_forward(const mote_layer_t* L, const void* x, 
   void* hs = base + pl.hs;
   auto* s = reinterpret_cast<float*>(base + pl.s);
 
+  auto* status = reinterpret_cast<uint32_t*>(base + pl.status);
   auto* tiles_routed = reinterpret_cast<int4*>(base + pl.tiles_routed);
   auto* tiles_shared = reinterpret_cast<int4*>(base + pl.tiles_shared);
-  auto* status = reinterpret_cast<uint32_t*>(base + pl.status);
   const int max_mtiles_routed = (int)(P / 128 + E);
   const int max_mtiles_shared = (int)((T + 127) / 128);
 
   const bool tensor_ok = (d % 128 == 0) && (f % 128 == 0);
+  const bool stream_ok = decode_stream_supported(d, f, E, k, T);
   int path = L->path;
-  if (path == MOTE_PATH_AUTO) path = tensor_ok ? MOTE_PATH_TENSOR : MOTE_PATH_SIMT;
-  if (path == MOTE_PATH_STREAM) return MOTE_ERR_SHAPE;   // not available yet
+  if (path == MOTE_PATH_AUTO) path = stream_ok ? MOTE_PATH_STREAM : tensor_ok ? MOTE_PATH_TENSOR : MOTE_PATH_SIMT;
+  if (path == MOTE_PATH_STREAM && !stream_ok) return MOTE_ERR_SHAPE;
   if (path == MOTE_PATH_TENSOR && !tensor_ok) return MOTE_ERR_SHAPE;
   const bool tensor = (path == MOTE_PATH_TENSOR);
-  const int interleave = tensor ? 1 : 0;
+  const int interleave = (tensor || path == MOTE_PATH_STREAM) ? 1 : 0;
+
+  if (path == MOTE_PATH_STREAM) {
+    // status word and the prologue's arrival counter
+    MOTE_CUDA_OK(cudaMemsetAsync(status, 0, 8, stream));
+    stage_mark(0, stream);
+    DecodeStreamArgs ds{};
+    ds.x = x; ds.T = T; ds.d = d; ds.f = f; ds.E = E; ds.k = k; ds.norm_topk = L->norm_topk;
+    ds.Wr = L->Wr; ds.router_bias = L->router_bias;
+    ds.gate_packed = L->gate_packed; ds.up_packed = L->up_packed; ds.down_packed = L->down_packed;
+    ds.alpha_gate = L->alpha_gate; ds.alpha_up = L->alpha_up; ds.alpha_down = L->alpha_down;
+    ds.sh_gate = L->sh_gate; ds.sh_up = L->sh_up; ds.sh_down = L->sh_down;
+    ds.topk_idx = topk_idx; ds.topk_w = topk_w; ds.offsets = offsets; ds.perm = perm; ds.inv = inv;
+    ds.qx = qx; ds.beta_x = beta_x; ds.rowsum_x = rowsum_x; ds.h = h; ds.qh = qh; ds.beta_h = beta_h;
+    ds.rowsum_h = rowsum_h; ds.y = y; ds.hs = hs; ds.s = s; ds.counter = status + 1;
+    ds.tap_gate = taps ? taps->acc_gate : nullptr; ds.tap_up = taps ? taps->acc_up : nullptr;
+    ds.tap_down = taps ? taps->acc_down : nullptr;
+    if (taps && (!taps->acc_gate != !taps->acc_up)) return MOTE_ERR_NULL;
+    mote_status_t st = launch_decode_stream(ds, 0, stream);   // Q_a(x), router, dispatch in one kernel
+    if (st) return st;
+    stage_mark(1, stream); stage_mark(2, stream); stage_mark(3, stream);
+    st = launch_decode_stream(ds, 1, stream);                 // routed and shared gate/up
+    if (st) return st;
+    stage_mark(4, stream);
+    st = launch_quant_rows_known_beta(h, P, f, qh, beta_h, rowsum_h, 1, stream);
+    if (st) return st;
+    stage_mark(5, stream);
+    st = launch_decode_stream(ds, 2, stream);                 // routed and shared down
+    if (st) return st;
+    stage_mark(6, stream); stage_mark(7, stream); stage_mark(8, stream);
+    st = launch_combine(s, y, topk_w, perm, residual, T, d, k, out, stream);
+    if (st) return st;
+    stage_mark(9, stream);
+    if (taps) {
+      auto d2d = [&](void* dst, const void* src, size_t bytes) -> bool {
+        return !dst || cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToDevice, stream) == cudaSuccess;
+      };
+      bool ok = d2d(taps->topk_idx, topk_idx, P * 4) && d2d(taps->topk_w, topk_w, P * 4) &&
+                d2d(taps->offsets, offsets, size_t(E + 1) * 4) && d2d(taps->perm, perm, P * 4) &&
+                d2d(taps->beta_x, beta_x, size_t(T) * 4) && d2d(taps->h_bf16, h, size_t(P) * f * 2) &&
+                d2d(taps->beta_h, beta_h, P * 4) && d2d(taps->y, y, size_t(P) * d * 4) &&
+                d2d(taps->shared_out, s, size_t(T) * d * 4);
+      if (!ok) return MOTE_ERR_CUDA;
+      if (taps->qx) {   // token order already; undo the k-interleave
+        copy_q_rows_kernel<<<148, 256, 0, stream>>>(qx, taps->qx, T, d / 16, nullptr, 0, 1);
+        MOTE_LAUNCH_OK();
+      }
+      if (taps->qh) {
+        copy_q_rows_kernel<<<148, 256, 0, stream>>>(qh, taps->qh, P, f / 16, nullptr, 0, 1);
+        MOTE_LAUNCH_OK();
+      }
+    }
+    return MOTE_OK;
+  }
 
   mote_status_t st;
   MOTE_CUDA_OK(cudaMemsetAsync(status, 0, 4, stream));

@@ -77,6 +77,25 @@ mote_status_t launch_shared_gateup_simt(const void* x, const void* Wg, const voi
 mote_status_t launch_shared_down_simt(const void* h, const void* Wd, int64_t T, int d, int f, float* s,
                                       cudaStream_t stream);
 
+// Decode path (T <= 64): prologue (Q_a(x), router, dispatch), streamed gate/up, Q_a(h), streamed
+// down.  Fills topk_*, offsets/perm/inv, qx (TOKEN order, k-interleaved), beta_x/rowsum_x (token
+// order), h, beta_h, qh, rowsum_h, y, hs, s; the caller runs the combine.
+struct DecodeStreamArgs {
+  const void* x; int64_t T; int d, f, E, k, norm_topk;
+  const float* Wr; const float* router_bias;
+  const uint8_t* gate_packed; const uint8_t* up_packed; const uint8_t* down_packed;
+  const float* alpha_gate; const float* alpha_up; const float* alpha_down;
+  const void* sh_gate; const void* sh_up; const void* sh_down;
+  int32_t* topk_idx; float* topk_w; int32_t* offsets; int32_t* perm; int32_t* inv;
+  int8_t* qx; float* beta_x; int32_t* rowsum_x;
+  void* h; int8_t* qh; float* beta_h; int32_t* rowsum_h; float* y; void* hs; float* s;
+  uint32_t* counter;                       // one zeroed word
+  int32_t* tap_gate; int32_t* tap_up; int32_t* tap_down;   // optional
+};
+bool decode_stream_supported(int d, int f, int E, int k, int64_t T);
+// phase 0: prologue, 1: gate/up (routed + shared), 2: down (routed + shared); Q_a(h) runs between 1 and 2
+mote_status_t launch_decode_stream(const DecodeStreamArgs& a, int phase, cudaStream_t stream);
+
 // out = [residual +] s + sum_j w_j * y[perm[t*k+j]]
 mote_status_t launch_combine(const float* s, const float* y, const float* w, const int32_t* perm,
                              const void* residual, int64_t T, int d, int k, void* out_bf16,

@@ -10,8 +10,9 @@ from parity_utils import bf16_bits, bf16_tensor, check_forward, check_packed_lay
 
 pytestmark = pytest.mark.gpu
 
-SIMT, TENSOR = 1, 2
+SIMT, TENSOR, STREAM = 1, 2, 3
 BOTH = [pytest.param(SIMT, id="simt"), pytest.param(TENSOR, id="tensor")]
+ALL = BOTH + [pytest.param(STREAM, id="stream")]
 
 
 @pytest.fixture(scope="module")
@@ -27,7 +28,7 @@ def _setup(mote, wl, path=1):
     return master, layer_or, layer_gpu
 
 
-@pytest.mark.parametrize("path", BOTH)
+@pytest.mark.parametrize("path", ALL)
 def test_c1_full_parity(mote, path):
     wl = synth.WORKLOADS["c1"]
     master, layer_or, layer_gpu = _setup(mote, wl, path)
@@ -48,6 +49,12 @@ def test_c1_full_parity(mote, path):
     (128, 256, 8, 2, 77, dict(bias="zipf"), TENSOR),
     (128, 384, 4, 1, 130, dict(norm_topk=0), TENSOR),     # down projection with 128-wide tiles
     (384, 640, 3, 3, 515, {}, TENSOR),                    # k = E, several row tiles per expert
+    (64, 128, 3, 3, 5, {}, STREAM),                       # k = E, one short reduction step
+    (128, 192, 2, 1, 1, {}, STREAM),                      # one token
+    (896, 4864, 4, 2, 17, dict(outlier_frac=0.01), STREAM),   # d/4 = 224 bytes: a ragged last step
+    (256, 512, 4, 2, 64, dict(bias="zipf"), STREAM),      # the largest batch, uneven expert loads
+    (192, 320, 8, 1, 33, dict(norm_topk=0), STREAM),
+    (128, 256, 64, 8, 37, {}, STREAM),                    # many experts, k = 8
 ])
 def test_small_shapes(mote, d, f, E, k, T, kw, path):
     wl = synth.custom("small", d, f, E, k, T, 2000 + d + f + T, **kw)
@@ -84,6 +91,34 @@ def test_run_to_run_determinism_and_token_permutation(mote, path):
     assert torch.equal(c, a[pm])
 
 
+def test_stream_path_idle_experts_residual_determinism(mote):
+    wl = synth.custom("skew", 128, 256, 4, 2, 40, 3003)
+    master = synth.master_layer(wl)
+    master["router_bias"] = np.array([50.0, -50.0, 40.0, -60.0], np.float32)   # experts 1 and 3 idle
+    layer_or = O.build_layer(master)
+    layer_gpu = mote.MoteLayer.from_master(master, path=STREAM)
+    x = synth.tokens(wl)
+    res = synth.tokens(wl, stream=1)
+    rep = check_forward(mote, layer_gpu, layer_or, x, residual_bits=res)
+    assert rep["counts"].tolist() == [40, 0, 40, 0]
+    rep2 = check_forward(mote, layer_gpu, layer_or, x, residual_bits=res, out_alias_residual=True)
+    assert torch.equal(rep["out"], rep2["out"])
+    xt = bf16_tensor(x)
+    pm = torch.randperm(wl.T, generator=torch.Generator().manual_seed(2)).cuda()
+    a = mote.mote_moe_forward(layer_gpu, xt).clone()
+    c = mote.mote_moe_forward(layer_gpu, xt[pm].contiguous())
+    assert torch.equal(c, a[pm])
+
+
+def test_stream_path_rejects_large_batches(mote):
+    wl = synth.custom("big", 128, 256, 4, 2, 65, 3004)
+    master = synth.master_layer(wl)
+    layer_gpu = mote.MoteLayer.from_master(master, path=STREAM)
+    with pytest.raises(mote.MoteError) as ei:
+        mote.mote_moe_forward(layer_gpu, bf16_tensor(synth.tokens(wl)))
+    assert ei.value.status == 2
+
+
 def test_zero_tokens_is_a_noop(mote):
     wl = synth.WORKLOADS["c1"]
     master, layer_or, layer_gpu = _setup(mote, wl)
@@ -92,7 +127,7 @@ def test_zero_tokens_is_a_noop(mote):
     assert out.shape == (0, wl.d)
 
 
-@pytest.mark.parametrize("path", BOTH)
+@pytest.mark.parametrize("path", ALL)
 @pytest.mark.parametrize("T", synth.C3_BATCHES)
 def test_c3_decode_batches(mote, T, path, c3_layers):
     wl, layer_or, layer_gpu = c3_layers
