@@ -78,13 +78,29 @@ struct ModeTraits {
   static constexpr bool kTernary = (MODE == MODE_T_GATEUP || MODE == MODE_T_DOWN);
   static constexpr bool kGateUp = (MODE == MODE_T_GATEUP || MODE == MODE_B_GATEUP);
   static constexpr int kStages = kTernary ? kStagesTernary : kStagesBf16;
-  static constexpr size_t kSmem =
-      1024 + size_t(kStages) * (kStageA + kStageB) + (kTernary ? size_t(kStagesP) * kStageP : 0) + sizeof(PipeBarriers);
+  // gate/up epilogue: every epilogue warp stages 32 rows x kEpiCols bf16 (row pitch padded by 16 B)
+  // and writes them out as whole row segments
+  // (bf16 gate/up only.  For the ternary gate/up, whose epilogue competes with the unpackers for
+  // issue slots, staging -- with plain stores or with a TMA store -- measured slower than letting
+  // every thread write its own 32 bytes.)
+  static constexpr int kEpiCols = 32;
+  static constexpr int kEpiPitch = kEpiCols * 2 + 16;
+  static constexpr size_t kEpiStage = (kGateUp && !kTernary) ? size_t(8) * 32 * kEpiPitch : 0;
+  static constexpr size_t kSmem = 1024 + size_t(kStages) * (kStageA + kStageB) +
+                                  (kTernary ? size_t(kStagesP) * kStageP : 0) + kEpiStage + sizeof(PipeBarriers);
 };
 
+// Item order.  The CTAs of the grid work on neighbouring items at the same time, and the operand
+// those items share is the one L2 serves to all of them from a single HBM read.
+//   gate/up: row tile fastest -- concurrent items share the (small) weight tile; the token operand
+//            (T x d) stays in L2 across column tiles;
+//   down:    column tile fastest -- concurrent items share the token operand (P x f, larger than
+//            L2 for long prefills), which is then read from HBM once instead of once per column tile.
+template <bool kGateUp>
 __device__ __forceinline__ void decode_item(const UmmaArgs& a, int item, int n_mtiles, int4& tile, int& n_tile) {
-  const int m_tile = item % n_mtiles;
-  n_tile = item / n_mtiles;
+  int m_tile;
+  if (kGateUp) { m_tile = item % n_mtiles; n_tile = item / n_mtiles; }
+  else { m_tile = item / a.n_ntiles; n_tile = item % a.n_ntiles; }
   tile = a.tiles[1 + m_tile];
 }
 
@@ -103,7 +119,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
   const uint32_t sP = sB + S * kStageB;
   uint8_t* genB = smem_gen + S * kStageA;
   uint8_t* genP = genB + S * kStageB;
-  PipeBarriers* bars = reinterpret_cast<PipeBarriers*>(genP + (TR::kTernary ? kStagesP * kStageP : 0));
+  uint8_t* genE = genP + (TR::kTernary ? kStagesP * kStageP : 0);
+  PipeBarriers* bars = reinterpret_cast<PipeBarriers*>(genE + TR::kEpiStage);
   volatile int* abort_flag = &bars->abort_flag;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -144,7 +161,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
       bool ok = true;
       for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x) {
         int4 tile; int n_tile;
-        decode_item(a, item, n_mtiles, tile, n_tile);
+        decode_item<TR::kGateUp>(a, item, n_mtiles, tile, n_tile);
         const int b_row = (a.b_rows_per_expert ? tile.x * a.b_rows_per_expert : 0) + n_tile * (TR::kGateUp ? a.bn / 2 : a.bn);
         for (int ks = 0; ks < a.k_steps; ++ks) {
           if (!(ok = mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1, abort_flag))) break;
@@ -174,7 +191,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
       bool ok = true;
       for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x) {
         int4 tile; int n_tile;
-        decode_item(a, item, n_mtiles, tile, n_tile);
+        decode_item<TR::kGateUp>(a, item, n_mtiles, tile, n_tile);
         const int b_row = tile.x * a.b_rows_per_expert + n_tile * (TR::kGateUp ? a.bn / 2 : a.bn);
         for (int ks = 0; ks < a.k_steps; ++ks) {
           if (!(ok = mbar_wait(smem_u32(&bars->empty_p[stage]), phase ^ 1, abort_flag))) break;
@@ -280,7 +297,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
     bool ok = true;
     for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x, ++local) {
       int4 tile; int n_tile;
-      decode_item(a, item, n_mtiles, tile, n_tile);
+      decode_item<TR::kGateUp>(a, item, n_mtiles, tile, n_tile);
       const int buf = local & 1;
       const uint32_t use = (uint32_t)(local >> 1);
       ok = mbar_wait(smem_u32(&bars->tmem_full[buf]), use & 1, abort_flag);
@@ -302,52 +319,78 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
         const int col0 = n_tile * 128;
         const bool row_fast = __fmul_rn(c0, c1) > 1e-12f;
         float hmax = 0.0f;                           // max |h| (before the bf16 rounding, which is monotonic)
+        constexpr int kCols = TR::kEpiCols, kPitch = TR::kEpiPitch;
+        constexpr int kLanesPerRow = kCols * 2 / 16, kRowsPerStore = 32 / kLanesPerRow;
+        uint8_t* stg = genE + (warp - 12) * 32 * kPitch;
 #pragma unroll 1
-        for (int c = chalf * 64; c < chalf * 64 + 64; c += 16) {
-          uint32_t rg[16], ru[16];
-          tmem_ld_32x32b_x16(t_row + c, rg);
-          tmem_ld_32x32b_x16(t_row + 128 + c, ru);
-          tmem_wait_ld();
-          if (row_ok) {
-            float hv[16];
-            if (TR::kTernary) {
-              uint32_t redo_mask = 0u;
+        for (int cr = chalf * 64; cr < chalf * 64 + 64; cr += kCols) {
+#pragma unroll 1
+          for (int c = cr; c < cr + kCols; c += 16) {
+            uint32_t rg[16], ru[16];
+            tmem_ld_32x32b_x16(t_row + c, rg);
+            tmem_ld_32x32b_x16(t_row + 128 + c, ru);
+            tmem_wait_ld();
+            if (row_ok) {
+              float hv[16];
+              if (TR::kTernary) {
+                uint32_t redo_mask = 0u;
 #pragma unroll
-              for (int j = 0; j < 16; ++j) {
-                bool redo;
-                hv[j] = glu_h_fast((int)rg[j] - rs, (int)ru[j] - rs, c0, c1, redo);
-                if (redo) redo_mask |= 1u << j;
+                for (int j = 0; j < 16; ++j) {
+                  bool redo;
+                  hv[j] = glu_h_fast((int)rg[j] - rs, (int)ru[j] - rs, c0, c1, redo);
+                  if (redo) redo_mask |= 1u << j;
+                }
+                if (!row_fast) redo_mask = 0xFFFFu;
+                if (redo_mask) {
+#pragma unroll
+                  for (int j = 0; j < 16; ++j)
+                    if ((redo_mask >> j) & 1u) hv[j] = glu_h((int)rg[j] - rs, (int)ru[j] - rs, c0, c1);
+                }
+#pragma unroll
+                for (int j = 0; j < 16; ++j) hmax = fmaxf(hmax, fabsf(hv[j]));
+              } else {
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                  const float g = __uint_as_float(rg[j]);
+                  hv[j] = __uint_as_float(ru[j]) * __fdividef(g, 1.0f + __expf(-g));
+                }
               }
-              if (!row_fast) redo_mask = 0xFFFFu;
-              if (redo_mask) {
+              uint32_t packed[8];
 #pragma unroll
-                for (int j = 0; j < 16; ++j)
-                  if ((redo_mask >> j) & 1u) hv[j] = glu_h((int)rg[j] - rs, (int)ru[j] - rs, c0, c1);
+              for (int j = 0; j < 8; ++j) packed[j] = pack_bf16x2(hv[2 * j], hv[2 * j + 1]);
+              if (TR::kTernary) {
+                uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<uint16_t*>(a.out) + row * a.n_out + col0 + c);
+                dst[0] = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+                dst[1] = make_uint4(packed[4], packed[5], packed[6], packed[7]);
+              } else {
+                uint4* sdst = reinterpret_cast<uint4*>(stg + lane * kPitch + (c - cr) * 2);
+                sdst[0] = make_uint4(packed[0], packed[1], packed[2], packed[3]);
+                sdst[1] = make_uint4(packed[4], packed[5], packed[6], packed[7]);
               }
+              if (TR::kTernary && a.tap0) {
+                int4* t0 = reinterpret_cast<int4*>(a.tap0 + row * a.n_out + col0 + c);
+                int4* t1 = reinterpret_cast<int4*>(a.tap1 + row * a.n_out + col0 + c);
 #pragma unroll
-              for (int j = 0; j < 16; ++j) hmax = fmaxf(hmax, fabsf(hv[j]));
-            } else {
-#pragma unroll
-              for (int j = 0; j < 16; ++j) {
-                const float g = __uint_as_float(rg[j]);
-                hv[j] = __uint_as_float(ru[j]) * __fdividef(g, 1.0f + __expf(-g));
+                for (int v = 0; v < 4; ++v) {
+                  t0[v] = make_int4((int)rg[4 * v] - rs, (int)rg[4 * v + 1] - rs, (int)rg[4 * v + 2] - rs, (int)rg[4 * v + 3] - rs);
+                  t1[v] = make_int4((int)ru[4 * v] - rs, (int)ru[4 * v + 1] - rs, (int)ru[4 * v + 2] - rs, (int)ru[4 * v + 3] - rs);
+                }
               }
             }
-            uint32_t packed[8];
+          }
+          if (!TR::kTernary) {
+            __syncwarp();
+            // the warp's 32 rows x kCols columns leave as whole row segments (kCols * 2 bytes each)
 #pragma unroll
-            for (int j = 0; j < 8; ++j) packed[j] = pack_bf16x2(hv[2 * j], hv[2 * j + 1]);
-            uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<uint16_t*>(a.out) + row * a.n_out + col0 + c);
-            dst[0] = make_uint4(packed[0], packed[1], packed[2], packed[3]);
-            dst[1] = make_uint4(packed[4], packed[5], packed[6], packed[7]);
-            if (TR::kTernary && a.tap0) {
-              int4* t0 = reinterpret_cast<int4*>(a.tap0 + row * a.n_out + col0 + c);
-              int4* t1 = reinterpret_cast<int4*>(a.tap1 + row * a.n_out + col0 + c);
-#pragma unroll
-              for (int v = 0; v < 4; ++v) {
-                t0[v] = make_int4((int)rg[4 * v] - rs, (int)rg[4 * v + 1] - rs, (int)rg[4 * v + 2] - rs, (int)rg[4 * v + 3] - rs);
-                t1[v] = make_int4((int)ru[4 * v] - rs, (int)ru[4 * v + 1] - rs, (int)ru[4 * v + 2] - rs, (int)ru[4 * v + 3] - rs);
+            for (int r0 = 0; r0 < 32; r0 += kRowsPerStore) {
+              const int r = r0 + lane / kLanesPerRow, piece = lane % kLanesPerRow;
+              if (q * 32 + r < tile.z) {
+                const uint4 v = *reinterpret_cast<const uint4*>(stg + r * kPitch + piece * 16);
+                uint16_t* orow = reinterpret_cast<uint16_t*>(a.out) + (int64_t(tile.y) + q * 32 + r) * a.n_out + col0 + cr;
+                reinterpret_cast<uint4*>(orow)[piece] = v;
               }
             }
+            __syncwarp();
           }
         }
         // bits of non-negative floats order like unsigned integers; bf16_rn(max) = max(bf16_rn)
