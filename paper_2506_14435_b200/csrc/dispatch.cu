@@ -4,13 +4,15 @@
 //   inv[P]        sorted row        ->  pair
 // Inside an expert the pairs keep their (token, slot) order, so the result does not depend on
 // thread scheduling.  One CTA walks the pairs in chunks of 1024; inside a chunk the rank of a
-// pair among equal experts comes from a warp-level match/popc prefix plus a per-warp histogram.
+// pair among equal experts comes from a warp-level match/popc prefix plus a per-warp histogram
+// that is turned into per-warp bases by a shuffle scan over the warps (one expert per warp).
 #include "mote_common.cuh"
 #include "mote_internal.h"
 
 namespace mote {
 
 constexpr int kDispatchThreads = 1024;
+constexpr int kBatch = 8;                 // chunks whose loads are issued together
 
 __global__ void __launch_bounds__(kDispatchThreads) dispatch_kernel(const int32_t* __restrict__ idx, int P, int E,
                                                                     int32_t* __restrict__ offsets,
@@ -21,14 +23,26 @@ __global__ void __launch_bounds__(kDispatchThreads) dispatch_kernel(const int32_
   __shared__ int s_count[MOTE_MAX_EXPERTS];
   __shared__ int s_running[MOTE_MAX_EXPERTS];
   __shared__ int s_warp[32][MOTE_MAX_EXPERTS];
+  __shared__ int s_pref[32][MOTE_MAX_EXPERTS];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
   if (tid < MOTE_MAX_EXPERTS) s_count[tid] = 0;
   for (int i = tid; i < 32 * MOTE_MAX_EXPERTS; i += kDispatchThreads) (&s_warp[0][0])[i] = 0;
   __syncthreads();
-  for (int p = tid; p < P; p += kDispatchThreads) {
-    const int e = idx[p];
-    if (e >= 0 && e < E) atomicAdd(&s_count[e], 1);
+  // histogram, one atomic per warp and expert; the loads of a batch are independent of each other
+  for (int base = 0; base < P; base += kBatch * kDispatchThreads) {
+    int ev[kBatch];
+#pragma unroll
+    for (int c = 0; c < kBatch; ++c) {
+      const int p = base + c * kDispatchThreads + tid;
+      ev[c] = p < P ? idx[p] : -1;
+    }
+#pragma unroll
+    for (int c = 0; c < kBatch; ++c) {
+      const int e = (ev[c] >= 0 && ev[c] < E) ? ev[c] : -1;
+      const unsigned peers = __match_any_sync(0xffffffffu, e);
+      if (e >= 0 && lane == __ffs(peers) - 1) atomicAdd(&s_count[e], __popc(peers));
+    }
   }
   __syncthreads();
   if (tid == 0) {
@@ -57,30 +71,44 @@ __global__ void __launch_bounds__(kDispatchThreads) dispatch_kernel(const int32_
   }
   __syncthreads();
 
-  for (int base = 0; base < P; base += kDispatchThreads) {
-    const int p = base + tid;
-    int e = -1;
-    if (p < P) {
-      e = idx[p];
-      if (e < 0 || e >= E) e = -1;
+  // s_warp[w][e]: pairs of expert e held by warp w in the current chunk (zero between chunks)
+  for (int base0 = 0; base0 < P; base0 += kBatch * kDispatchThreads) {
+    int ev[kBatch];
+#pragma unroll
+    for (int c = 0; c < kBatch; ++c) {
+      const int p = base0 + c * kDispatchThreads + tid;
+      ev[c] = p < P ? idx[p] : -1;
     }
-    const unsigned peers = __match_any_sync(0xffffffffu, e);
-    const int rank = __popc(peers & ((1u << lane) - 1u));
-    if (e >= 0 && rank == 0) s_warp[warp][e] = __popc(peers);
-    __syncthreads();
-    if (e >= 0) {
-      int pos = s_running[e] + rank;
-      for (int w = 0; w < warp; ++w) pos += s_warp[w][e];
-      perm[p] = pos;
-      inv[pos] = p;
+#pragma unroll
+    for (int c = 0; c < kBatch; ++c) {
+      if (base0 + c * kDispatchThreads >= P) break;            // uniform over the CTA
+      const int p = base0 + c * kDispatchThreads + tid;
+      const int e = (ev[c] >= 0 && ev[c] < E) ? ev[c] : -1;
+      const unsigned peers = __match_any_sync(0xffffffffu, e);
+      const int rank = __popc(peers & ((1u << lane) - 1u));
+      if (e >= 0 && rank == 0) s_warp[warp][e] = __popc(peers);
+      __syncthreads();
+      // exclusive scan over the 32 warps, one expert per warp and round (lane = warp index)
+      for (int ee = warp; ee < E; ee += 32) {
+        const int v = s_warp[lane][ee];
+        s_warp[lane][ee] = 0;
+        int incl = v;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int n = __shfl_up_sync(0xffffffffu, incl, o);
+          if (lane >= o) incl += n;
+        }
+        const int first = s_running[ee];
+        s_pref[lane][ee] = first + incl - v;
+        if (lane == 31) s_running[ee] = first + incl;
+      }
+      __syncthreads();
+      if (e >= 0) {
+        const int pos = s_pref[warp][e] + rank;
+        perm[p] = pos;
+        inv[pos] = p;
+      }
     }
-    __syncthreads();
-    if (tid < E) {
-      int add = 0;
-      for (int w = 0; w < 32; ++w) { add += s_warp[w][tid]; s_warp[w][tid] = 0; }
-      s_running[tid] += add;
-    }
-    __syncthreads();
   }
 }
 

@@ -292,18 +292,26 @@ extern "C" mote_status_t mote_moe_forward(const mote_layer_t* L, const void* x, 
   stage_mark(6, stream);
   // S7 shared expert
   st = tensor ? launch_shared_umma(x, L->sh_gate, L->sh_up, true, T, d, f, hs, tiles_shared, max_mtiles_shared,
-                                   status, stream)
+                                   status, nullptr, stream)
               : launch_shared_gateup_simt(x, L->sh_gate, L->sh_up, T, d, f, hs, stream);
   if (st) return st;
   stage_mark(7, stream);
-  st = tensor ? launch_shared_umma(hs, L->sh_down, nullptr, false, T, f, d, s, tiles_shared, max_mtiles_shared,
-                                   status, stream)
-              : launch_shared_down_simt(hs, L->sh_down, T, d, f, s, stream);
-  if (st) return st;
-  stage_mark(8, stream);
-  // S8 combine
-  st = launch_combine(s, y, topk_w, perm, residual, T, d, k, out, stream);
-  if (st) return st;
+  if (tensor) {
+    // shared down projection with S8 (combine, residual, bf16 rounding) in its epilogue; the fp32
+    // shared output is written only when a tap asks for it
+    CombineArgs cb{y, topk_w, perm, residual, out, k};
+    st = launch_shared_umma(hs, L->sh_down, nullptr, false, T, f, d, (taps && taps->shared_out) ? s : nullptr,
+                            tiles_shared, max_mtiles_shared, status, &cb, stream);
+    if (st) return st;
+    stage_mark(8, stream);
+  } else {
+    st = launch_shared_down_simt(hs, L->sh_down, T, d, f, s, stream);
+    if (st) return st;
+    stage_mark(8, stream);
+    // S8 combine
+    st = launch_combine(s, y, topk_w, perm, residual, T, d, k, out, stream);
+    if (st) return st;
+  }
   stage_mark(9, stream);
 
   if (taps) {

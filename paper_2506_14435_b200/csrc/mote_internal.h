@@ -67,9 +67,14 @@ mote_status_t launch_ternary_umma(const TernaryGemmArgs& a, bool gateup, const i
 // writes q (k-interleaved if asked), the clamped beta in place, and accumulates rowsum (zeroed).
 mote_status_t launch_quant_rows_known_beta(const void* h_bf16, int64_t rows, int n, int8_t* q, float* beta,
                                            int32_t* rowsum, int interleave, cudaStream_t stream);
+// comb (down projection only, may be null): fold the combine of Eq. 2 / Eq. 4 into the epilogue and
+// write the layer output directly; `out` (fp32 s) may then be null.
+struct CombineArgs {
+  const float* y; const float* w; const int32_t* perm; const void* residual; void* out; int k;
+};
 mote_status_t launch_shared_umma(const void* act, const void* w0, const void* w1, bool gateup, int64_t T, int K,
                                  int N, void* out, const int4* tiles, int max_mtiles, uint32_t* status,
-                                 cudaStream_t stream);
+                                 const CombineArgs* comb, cudaStream_t stream);
 
 // CUDA-core bf16 GEMMs of the shared expert.
 mote_status_t launch_shared_gateup_simt(const void* x, const void* Wg, const void* Wu, int64_t T, int d,

@@ -7,8 +7,8 @@
 //   B_GATEUP  shared expert gate/up (Eq. 2): bf16 x bf16 -> fp32 -> h_shared bf16
 //   B_DOWN    shared expert down -> s fp32
 //
-// Tile: 128 token rows (UMMA M, one TMEM lane per row) x BN weight rows (UMMA N = 256, or 128 for
-// a down projection whose width is not a multiple of 256); K advances 128 bytes of the token
+// Tile: 128 token rows (UMMA M, one TMEM lane per row) x BN weight rows (UMMA N = 256; for a down
+// projection the largest multiple of 32 up to 256 that divides its width, e.g. 224 for 896); K advances 128 bytes of the token
 // operand per pipeline stage (128 int8 or 64 bf16), four K=32-byte MMAs per stage.
 //
 // Ternary weights travel as 2-bit codes all the way into shared memory (TMA box of 32 bytes per
@@ -65,6 +65,10 @@ struct UmmaArgs {
   int32_t* tap1;
   uint32_t* beta_out_bits;  // gate/up of the routed experts: running max |h| per row (atomicMax on the bits)
   uint32_t* status;
+  // shared down projection with the combine of Eq. 2 and Eq. 4 folded into its epilogue (comb_out != null):
+  //   comb_out[t, :] = bf16( s[t, :] + sum_j comb_w[t, j] * comb_y[comb_perm[t*k + j], :] [+ comb_res[t, :]] )
+  const float* comb_y; const float* comb_w; const int32_t* comb_perm; const uint16_t* comb_res; uint16_t* comb_out;
+  int comb_k;
 };
 
 struct __align__(8) PipeBarriers {
@@ -177,7 +181,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
               tma_load_2d(sB + stage * kStageB + 128 * 128, &tm_b1, ks * 64, b_row, bar);
             } else {
               tma_load_2d(sB + stage * kStageB, &tm_b0, ks * 64, b_row, bar);
-              if (a.bn == 256) tma_load_2d(sB + stage * kStageB + 128 * 128, &tm_b0, ks * 64, b_row + 128, bar);
+              if (a.bn > 128) tma_load_2d(sB + stage * kStageB + 128 * 128, &tm_b1, ks * 64, b_row + 128, bar);
             }
           }
           if (++stage == S) { stage = 0; phase ^= 1; }
@@ -203,7 +207,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
             tma_load_2d(dst + 128 * 32, &tm_b1, ks * 32, b_row, bar);
           } else {
             tma_load_2d(dst, &tm_b0, ks * 32, b_row, bar);
-            if (a.bn == 256) tma_load_2d(dst + 128 * 32, &tm_b0, ks * 32, b_row + 128, bar);
+            if (a.bn > 128) tma_load_2d(dst + 128 * 32, &tm_b1, ks * 32, b_row + 128, bar);
           }
           if (++stage == kStagesP) { stage = 0; phase ^= 1; }
         }
@@ -250,7 +254,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
       const int tid = (threadIdx.x - 128) & 127;
       uint32_t stage = 0, phase = 0, pstage = 0, pphase = 0, step = 0;
       bool ok = true;
-      const int chunks_per_thread = a.bn / 64;       // bn*2 chunks of 16 packed bytes over 128 threads
+      const int n_chunks = a.bn * 2;                 // chunks of 16 packed bytes, spread over 128 threads
       for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x) {
         for (int ks = 0; ks < a.k_steps; ++ks, ++step) {
           if ((step & 1u) == (uint32_t)group) {
@@ -260,8 +264,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
             if (!ok) break;
             const uint8_t* src = genP + pstage * kStageP;
             uint8_t* dst = genB + stage * kStageB;
-            for (int i = 0; i < chunks_per_thread; ++i) {
-              const int c = i * 128 + tid;
+            for (int c = tid; c < n_chunks; c += 128) {
               const int r = c >> 1, half = c & 1;
               const uint4 w = *reinterpret_cast<const uint4*>(src + c * 16);
               const uint32_t pw[4] = {w.x, w.y, w.z, w.w};
@@ -401,32 +404,67 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
       } else {
         const int col0 = n_tile * a.bn;
         const int cbeg = chalf * (a.bn / 2), cend = cbeg + a.bn / 2;
+        const bool combine = !TR::kTernary && a.comb_out != nullptr;
+        float cw[MOTE_MAX_TOPK];
+        const float* cy[MOTE_MAX_TOPK];
+        if (combine && row_ok) {
+#pragma unroll
+          for (int j = 0; j < MOTE_MAX_TOPK; ++j)
+            if (j < a.comb_k) {
+              cw[j] = a.comb_w[row * a.comb_k + j];
+              cy[j] = a.comb_y + int64_t(a.comb_perm[row * a.comb_k + j]) * a.n_out + col0;
+            }
+        }
 #pragma unroll 1
         for (int c = cbeg; c < cend; c += 16) {
           uint32_t ra[16];
           tmem_ld_32x32b_x16(t_row + c, ra);
           tmem_wait_ld();
           if (row_ok) {
-            float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(a.out) + row * a.n_out + col0 + c);
+            float o[16];
 #pragma unroll
-            for (int v = 0; v < 4; ++v) {
-              float4 o;
-              if (TR::kTernary) {
-                o.x = __fmul_rn(i2f_small((int)ra[4 * v] - rs), c0);
-                o.y = __fmul_rn(i2f_small((int)ra[4 * v + 1] - rs), c0);
-                o.z = __fmul_rn(i2f_small((int)ra[4 * v + 2] - rs), c0);
-                o.w = __fmul_rn(i2f_small((int)ra[4 * v + 3] - rs), c0);
-              } else {
-                o = make_float4(__uint_as_float(ra[4 * v]), __uint_as_float(ra[4 * v + 1]),
-                                __uint_as_float(ra[4 * v + 2]), __uint_as_float(ra[4 * v + 3]));
-              }
-              dst[v] = o;
+            for (int v = 0; v < 16; ++v)
+              o[v] = TR::kTernary ? __fmul_rn(i2f_small((int)ra[v] - rs), c0) : __uint_as_float(ra[v]);
+            if (a.out) {
+              float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(a.out) + row * a.n_out + col0 + c);
+#pragma unroll
+              for (int v = 0; v < 4; ++v) dst[v] = make_float4(o[4 * v], o[4 * v + 1], o[4 * v + 2], o[4 * v + 3]);
             }
             if (TR::kTernary && a.tap0) {
               int4* t0 = reinterpret_cast<int4*>(a.tap0 + row * a.n_out + col0 + c);
 #pragma unroll
               for (int v = 0; v < 4; ++v)
                 t0[v] = make_int4((int)ra[4 * v] - rs, (int)ra[4 * v + 1] - rs, (int)ra[4 * v + 2] - rs, (int)ra[4 * v + 3] - rs);
+            }
+            if (combine) {
+              // fp32, slots in ascending j, then the residual, one bf16 rounding
+#pragma unroll
+              for (int j = 0; j < MOTE_MAX_TOPK; ++j)
+                if (j < a.comb_k) {
+                  const float4* yp = reinterpret_cast<const float4*>(cy[j] + c);
+#pragma unroll
+                  for (int v = 0; v < 4; ++v) {
+                    const float4 yv = yp[v];
+                    o[4 * v] = fmaf(cw[j], yv.x, o[4 * v]);         o[4 * v + 1] = fmaf(cw[j], yv.y, o[4 * v + 1]);
+                    o[4 * v + 2] = fmaf(cw[j], yv.z, o[4 * v + 2]); o[4 * v + 3] = fmaf(cw[j], yv.w, o[4 * v + 3]);
+                  }
+                }
+              if (a.comb_res) {
+                const uint4* rp = reinterpret_cast<const uint4*>(a.comb_res + row * a.n_out + col0 + c);
+#pragma unroll
+                for (int v = 0; v < 2; ++v) {
+                  const uint4 r = rp[v];
+                  const uint32_t rw[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+                  for (int u = 0; u < 4; ++u) { o[8 * v + 2 * u] += bf16_lo(rw[u]); o[8 * v + 2 * u + 1] += bf16_hi(rw[u]); }
+                }
+              }
+              uint32_t pk[8];
+#pragma unroll
+              for (int v = 0; v < 8; ++v) pk[v] = f32_to_bf16_bits(o[2 * v]) | (f32_to_bf16_bits(o[2 * v + 1]) << 16);
+              uint4* od = reinterpret_cast<uint4*>(a.comb_out + row * a.n_out + col0 + c);
+              od[0] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+              od[1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
             }
           }
         }
@@ -486,6 +524,14 @@ static bool make_map_2d(CUtensorMap* m, const void* base, CUtensorMapDataType dt
             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Width of a down-projection tile: the largest multiple of 32 up to 256 that divides N (N is a
+// multiple of 128).  Wider tiles reuse the token operand for more MMA work per byte fetched.
+static int pick_bn(int N) {
+  for (int bn = 256; bn > 128; bn -= 32)
+    if (N % bn == 0) return bn;
+  return 128;
+}
+
 template <int MODE>
 static mote_status_t launch_umma(const CUtensorMap& ta, const CUtensorMap& tb0, const CUtensorMap& tb1,
                                  const UmmaArgs& a, int max_items, cudaStream_t stream) {
@@ -510,15 +556,16 @@ mote_status_t launch_ternary_umma(const TernaryGemmArgs& g, bool gateup, const i
                                   cudaStream_t stream) {
   if (g.P == 0) return MOTE_OK;
   CUtensorMap ta, tb0, tb1;
-  const int bn = gateup ? 256 : ((g.N % 256 == 0) ? 256 : 128);
+  const int bn = gateup ? 256 : pick_bn(g.N);
   if (!make_map_2d(&ta, g.qa, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)g.P, (uint64_t)g.K, 128, 128,
                    CU_TENSOR_MAP_SWIZZLE_128B))
     return MOTE_ERR_CUDA;
   if (!make_map_2d(&tb0, g.w0, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)g.E * g.N, (uint64_t)g.K / 4, 128, 32,
                    CU_TENSOR_MAP_SWIZZLE_NONE))
     return MOTE_ERR_CUDA;
+  // second map: the up matrix (gate/up), or the rows beyond 128 of a down tile
   if (!make_map_2d(&tb1, gateup ? g.w1 : g.w0, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)g.E * g.N,
-                   (uint64_t)g.K / 4, 128, 32, CU_TENSOR_MAP_SWIZZLE_NONE))
+                   (uint64_t)g.K / 4, (gateup || bn <= 128) ? 128 : bn - 128, 32, CU_TENSOR_MAP_SWIZZLE_NONE))
     return MOTE_ERR_CUDA;
   UmmaArgs a{};
   a.tiles = tiles;
@@ -539,18 +586,18 @@ mote_status_t launch_ternary_umma(const TernaryGemmArgs& g, bool gateup, const i
 
 mote_status_t launch_shared_umma(const void* act, const void* w0, const void* w1, bool gateup, int64_t T, int K,
                                  int N, void* out, const int4* tiles, int max_mtiles, uint32_t* status,
-                                 cudaStream_t stream) {
+                                 const CombineArgs* comb, cudaStream_t stream) {
   if (T == 0) return MOTE_OK;
   CUtensorMap ta, tb0, tb1;
-  const int bn = gateup ? 256 : ((N % 256 == 0) ? 256 : 128);
+  const int bn = gateup ? 256 : pick_bn(N);
   if (!make_map_2d(&ta, act, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)T, (uint64_t)K, 128, 64,
                    CU_TENSOR_MAP_SWIZZLE_128B))
     return MOTE_ERR_CUDA;
   if (!make_map_2d(&tb0, w0, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)N, (uint64_t)K, 128, 64,
                    CU_TENSOR_MAP_SWIZZLE_128B))
     return MOTE_ERR_CUDA;
-  if (!make_map_2d(&tb1, gateup ? w1 : w0, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)N, (uint64_t)K, 128, 64,
-                   CU_TENSOR_MAP_SWIZZLE_128B))
+  if (!make_map_2d(&tb1, gateup ? w1 : w0, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)N, (uint64_t)K,
+                   (gateup || bn <= 128) ? 128 : bn - 128, 64, CU_TENSOR_MAP_SWIZZLE_128B))
     return MOTE_ERR_CUDA;
   UmmaArgs a{};
   a.tiles = tiles;
@@ -561,6 +608,11 @@ mote_status_t launch_shared_umma(const void* act, const void* w0, const void* w1
   a.b_rows_per_expert = 0;
   a.out = out;
   a.status = status;
+  if (comb && !gateup) {
+    a.comb_y = comb->y; a.comb_w = comb->w; a.comb_perm = comb->perm;
+    a.comb_res = static_cast<const uint16_t*>(comb->residual); a.comb_out = static_cast<uint16_t*>(comb->out);
+    a.comb_k = comb->k;
+  }
   const int max_items = max_mtiles * a.n_ntiles;
   return gateup ? launch_umma<MODE_B_GATEUP>(ta, tb0, tb1, a, max_items, stream)
                 : launch_umma<MODE_B_DOWN>(ta, tb0, tb1, a, max_items, stream);
