@@ -96,15 +96,22 @@ class ClockSampler:
                 "samples": len(sm)}
 
 
-def build_gpu_layer(wl: synth.Workload, device):
-    import paper_2506_14435_b200 as mote
-    master = synth.master_layer(wl)
-    return mote, mote.MoteLayer.from_master(master, device=device), master
+# ncu dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the captures
+# summarised under profiles/ (null once the kernel has changed since, or where no capture exists)
+NCU_TRAFFIC_BYTES = {}
 
 
-def dominant_stage_work(wl: synth.Workload, stage: str, counts=None):
-    """Algorithmic work of one launch of a stage: (amount, kind) with kind 'int8' | 'bf16' | 'bytes'."""
+def stage_work(wl: synth.Workload, stage: str, stream_path: bool, experts_touched: float):
+    """Algorithmic work of one launch of a stage: (amount, kind), kind 'int8' | 'bf16' | 'bytes'.
+    On the decode path the gate/up and down stages each cover the routed AND the shared expert and
+    are bound by the weight bytes they stream: 2-bit codes of the experts that received tokens plus
+    the bf16 shared matrices."""
     P, T, d, f = wl.T * wl.k, wl.T, wl.d, wl.f
+    if stream_path:
+        if stage == "gateup_ternary":
+            return experts_touched * 2 * f * d / 4 + 2.0 * f * d * 2, "bytes"
+        if stage == "down_ternary":
+            return experts_touched * f * d / 4 + f * d * 2.0, "bytes"
     if stage == "gateup_ternary":
         return 2.0 * P * d * 2 * f, "int8"
     if stage == "down_ternary":
@@ -124,6 +131,22 @@ def dominant_stage_work(wl: synth.Workload, stage: str, counts=None):
     return P * 12.0, "bytes"
 
 
+def max_over_ranks(values, device, world: int):
+    """Every rank passes its own times; all get the slowest rank's (the job is as slow as that)."""
+    if world <= 1:
+        return list(values)
+    import torch.distributed as dist
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def job_tokens_per_s(world: int, tokens_per_rank: int, steps: int, total_ms: float) -> float:
+    """Whole-job throughput of `world` replicas, each processing its own batch (weak scaling, no
+    collective on the data path): all ranks' tokens over the slowest rank's time."""
+    return world * tokens_per_rank * steps / (total_ms * 1e-3)
+
+
 def run_ours(args):
     rank = int(os.environ.get("RANK", 0))
     local_rank = int(os.environ.get("LOCAL_RANK", 0))
@@ -136,16 +159,46 @@ def run_ours(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
     wl = parse_workload(args.workload)
-    mote, layer, master = build_gpu_layer(wl, dev)
+    import paper_2506_14435_b200 as mote
     from paper_2506_14435_b200.binding import mote_moe_forward_host, mote_moe_forward_profile
 
-    x_bits = synth.tokens(wl, stream=rank)
-    x_host = torch.from_numpy(x_bits.view(np.int16).copy()).view(torch.bfloat16).pin_memory()
+    n_layers = wl.n_layers if args.layers is None else args.layers
+    is_stack = wl.n_layers > 1
+    master = None
+    if is_stack:
+        # 36 layers of 0.8 G weights each: drawn on the device (minutes on the host); every layer distinct
+        layers = [mote.MoteLayer.from_device_draws(wl.d, wl.f, wl.E, wl.k, wl.norm_topk,
+                                                   synth.device_draw(wl, l, dev), device=dev) for l in range(n_layers)]
+        stack = mote.MoteStack(layers)
+        x = synth.device_tokens(wl, dev, stream=rank)
+        x_host = x.cpu().pin_memory()
+        x_bits = None
+    else:
+        master = synth.master_layer(wl)
+        layers = [mote.MoteLayer.from_master(master, device=dev)]
+        x_bits = synth.tokens(wl, stream=rank)
+        x_host = torch.from_numpy(x_bits.view(np.int16).copy()).view(torch.bfloat16).pin_memory()
+        x = x_host.to(dev)
     out_host = torch.empty_like(x_host).pin_memory()
-    x = x_host.to(dev)
     out = torch.empty_like(x)
     flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
     stream = torch.cuda.current_stream()
+    stream_path = wl.T <= 64 and wl.d % 64 == 0 and wl.f % 64 == 0
+
+    def step_device():
+        if is_stack:
+            mote.mote_stack_forward(stack, x, out=out)
+        else:
+            mote.mote_moe_forward(layers[0], x, out=out)
+
+    def step_host():
+        if is_stack:                                    # host buffers in and out around the C-ABI call
+            x.copy_(x_host, non_blocking=True)
+            mote.mote_stack_forward(stack, x, out=out)
+            out_host.copy_(out, non_blocking=True)
+            torch.cuda.synchronize()
+        else:
+            mote_moe_forward_host(layers[0], x_host, out_host)      # synchronises the stream itself
 
     def barrier():
         if world > 1:
@@ -164,15 +217,25 @@ def run_ours(args):
         torch.cuda.synchronize()
         return [s.elapsed_time(e) for s, e in zip(starts, ends)]
 
+    # experts that receive tokens (decides the decode path's algorithmic bytes), layer by layer
+    touched = []
+    cur = x
+    for layer in layers:
+        taps = layer.alloc_taps(wl.T, names=["offsets"])
+        nxt = mote.mote_moe_forward(layer, cur, residual=cur if is_stack else None, taps=taps)
+        touched.append(int((taps["offsets"][1:] - taps["offsets"][:-1] > 0).sum().item()))
+        cur = nxt
+    experts_touched = sum(touched) / len(touched)
+
     # ---- device-resident timing
     for _ in range(args.warmup):
-        mote.mote_moe_forward(layer, x, out=out)
+        step_device()
     launches_per_step = mote.lib.mote_last_launch_count()
     barrier()
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
-    per_step = timed_loop(lambda: mote.mote_moe_forward(layer, x, out=out), args.steps)
+    per_step = timed_loop(step_device, args.steps)
     barrier()
     total_ms = sum(per_step)
 
@@ -181,31 +244,34 @@ def run_ours(args):
     n_prof = max(3, min(args.steps, 10))
     for i in range(n_prof):
         flush.fill_(i)
-        ms = mote_moe_forward_profile(layer, x, out=out)
-        for k_, v in ms.items():
+        cur = x
+        tot = {}
+        for layer in layers:
+            nxt = torch.empty_like(cur)
+            ms = mote_moe_forward_profile(layer, cur, out=nxt, residual=cur if is_stack else None)
+            for k_, v in ms.items():
+                tot[k_] = tot.get(k_, 0.0) + v
+            cur = nxt
+        for k_, v in tot.items():
             stage_acc.setdefault(k_, []).append(v)
     clocks = sampler.stop() if rank == 0 else None
-    stage_ms = {k_: statistics.mean(v) for k_, v in stage_acc.items()}
+    stage_ms = {k_: statistics.mean(v) for k_, v in stage_acc.items()}     # summed over the layers
 
-    # ---- end to end through the host-buffer entry point
+    # ---- end to end: host buffers in and out
     for _ in range(min(args.warmup, 3)):
-        mote_moe_forward_host(layer, x_host, out_host)
+        step_host()
     barrier()
     e2e_ms = []
     for i in range(args.steps):
         flush.fill_(i & 0xFF)
         torch.cuda.synchronize()
         t0 = time.perf_counter()
-        mote_moe_forward_host(layer, x_host, out_host)      # synchronises the stream itself
+        step_host()
         e2e_ms.append((time.perf_counter() - t0) * 1e3)
     barrier()
     e2e_total = sum(e2e_ms)
 
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([total_ms, e2e_total], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, e2e_total = t.tolist()
+    total_ms, e2e_total = max_over_ranks([total_ms, e2e_total], dev, world)
     if rank != 0:
         if world > 1:
             import torch.distributed as dist
@@ -214,37 +280,48 @@ def run_ours(args):
 
     peaks = measured_peaks()
     ms_per_step = total_ms / args.steps
-    tokens_per_s = world * wl.T * args.steps / (total_ms * 1e-3)
+    tokens_per_s = job_tokens_per_s(world, wl.T, args.steps, total_ms)
     decode = wl.T <= 64
     dom = max(stage_ms, key=stage_ms.get)
-    work, kind = dominant_stage_work(wl, dom)
-    dur_s = stage_ms[dom] * 1e-3
+    work, kind = stage_work(wl, dom, stream_path, experts_touched)
+    dur_s = stage_ms[dom] * 1e-3 / len(layers)          # average duration of one launch of that kernel
     if kind == "bytes":
         roof = dict(bound="hbm", achieved=work / dur_s / 1e9, peak=peaks["hbm_gbs"], unit="GB/s")
     else:
         peak = peaks["bf16_tflops"] * (NOMINAL_INT8_OVER_BF16 if kind == "int8" else 1.0)
         roof = dict(bound="tensor", achieved=work / dur_s / 1e12, peak=peak, unit="TOP/s" if kind == "int8" else "TFLOP/s")
     roof["frac"] = roof["achieved"] / roof["peak"]
-    roof["traffic"] = None
+    roof["traffic"] = NCU_TRAFFIC_BYTES.get((wl.name if not decode else f"{wl.name}-{wl.T}", dom))
     roof["kernel"] = dom
-    roof["kernel_ms"] = stage_ms[dom]
+    roof["kernel_ms"] = dur_s * 1e3
+    roof["algorithmic_work_per_launch"] = work
     roof["peak_source"] = ("of measured" if peaks["source"] == "measured" else "of fallback") + \
         (" (bf16 burst x2 nominal int8:bf16 ratio)" if kind == "int8" else "")
-
+    weight_bytes = len(layers) * (experts_touched * 3 * wl.d * wl.f / 4 + 6.0 * wl.d * wl.f)
     line = {
         "metric": "MoTE layer tokens/sec (prefill)" if not decode else "MoTE layer tokens/sec (decode batch)",
         "value": tokens_per_s, "unit": "tokens/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": ms_per_step, "us_per_layer": ms_per_step * 1e3, "higher_is_better": True,
+        "ms_per_step": ms_per_step, "us_per_layer": ms_per_step * 1e3 / len(layers),
+        "us_per_token": ms_per_step * 1e3 / wl.T, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "int8xint2->int32 routed, bf16 shared", "data": "synthetic",
         "config": {"workload": wl.name, "d": wl.d, "f": wl.f, "E": wl.E, "k": wl.k, "T_per_gpu": wl.T,
+                   "layers": len(layers), "experts_touched_per_layer": experts_touched,
                    "l2": "flushed between timed iterations (512 MiB write)", "parallelism": f"replicas x{world}"},
         "stage_ms": stage_ms, "roofline": roof,
-        "e2e": {"value": world * wl.T * args.steps / (e2e_total * 1e-3), "unit": "tokens/s",
+        "weights_touched_gbs": weight_bytes / (ms_per_step * 1e-3) / 1e9,
+        "e2e": {"value": job_tokens_per_s(world, wl.T, args.steps, e2e_total), "unit": "tokens/s",
                 "h2d_bytes_per_step": int(x_host.numel() * 2), "d2h_bytes_per_step": int(out_host.numel() * 2)},
         "gpu_launches": launches_per_step * args.steps, "clocks": clocks,
     }
     if world == 1:
-        line["cpu_baseline"] = cpu_baseline(wl, master, x_bits, budget_s=20.0)
+        if is_stack:                                    # the oracle needs host-drawn weights: layer 0, scaled by the depth
+            master = synth.master_layer(wl)
+            x_bits = synth.tokens(wl)
+        cb = cpu_baseline(wl, master, x_bits, budget_s=20.0)
+        if is_stack:
+            cb["value"] /= len(layers)
+            cb["sample"] += f"; one layer timed, value divided by the {len(layers)} layers of the stack"
+        line["cpu_baseline"] = cb
     print(json.dumps(line))
     if world > 1:
         import torch.distributed as dist
@@ -303,6 +380,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="c2")
+    ap.add_argument("--layers", type=int, default=None, help="layers of a stacked workload (c5-T: default 36)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup

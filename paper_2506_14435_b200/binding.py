@@ -58,6 +58,11 @@ lib.mote_host_staging_bytes.argtypes = [C.c_int, C.c_int64]
 lib.mote_moe_forward.restype = C.c_int
 lib.mote_moe_forward.argtypes = [C.POINTER(mote_layer_t), C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p,
                                  C.POINTER(mote_taps_t), C.c_void_p, C.c_size_t, C.c_void_p]
+lib.mote_stack_workspace_bytes.restype = C.c_size_t
+lib.mote_stack_workspace_bytes.argtypes = [C.POINTER(mote_layer_t), C.c_int, C.c_int64]
+lib.mote_stack_forward.restype = C.c_int
+lib.mote_stack_forward.argtypes = [C.POINTER(mote_layer_t), C.c_int, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p,
+                                   C.c_void_p, C.c_size_t, C.c_void_p]
 lib.mote_moe_forward_host.restype = C.c_int
 lib.mote_moe_forward_host.argtypes = [C.POINTER(mote_layer_t), C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p,
                                       C.c_void_p, C.c_size_t, C.c_void_p]
@@ -189,6 +194,25 @@ class MoteLayer:
                    packed["gate"], packed["up"], packed["down"], alphas["gate"], alphas["up"], alphas["down"],
                    bf16(master["sh_gate"]), bf16(master["sh_up"]), bf16(master["sh_down"]), path=path)
 
+    @classmethod
+    def from_device_draws(cls, d, f, E, k, norm_topk, draw, device="cuda", path=PATH_AUTO):
+        """Offline step with weights that are already on the device: draw(name, expert) returns
+        fp32 CUDA matrices for "gate"/"up"/"down", bf16 ones for "sh_gate"/"sh_up"/"sh_down",
+        fp32 "Wr" and "bias" (or None); every routed matrix goes through mote_ternarize_pack."""
+        dev = torch.device(device)
+        packed, alphas = {}, {}
+        for name, shape in (("gate", (f, d)), ("up", (f, d)), ("down", (d, f))):
+            buf = torch.empty((E, shape[0], shape[1] // 4), dtype=torch.uint8, device=dev)
+            al = torch.empty(E, dtype=torch.float32, device=dev)
+            for e in range(E):
+                p, a = mote_ternarize_pack(draw(name, e).contiguous())
+                buf[e].copy_(p)
+                al[e:e + 1].copy_(a)
+            packed[name], alphas[name] = buf, al
+        return cls(d, f, E, k, norm_topk, draw("Wr").contiguous(), draw("bias"),
+                   packed["gate"], packed["up"], packed["down"], alphas["gate"], alphas["up"], alphas["down"],
+                   draw("sh_gate").contiguous(), draw("sh_up").contiguous(), draw("sh_down").contiguous(), path=path)
+
     def struct(self) -> mote_layer_t:
         t = self.tensors
         s = mote_layer_t(self.d, self.f, self.E, self.k, self.norm_topk, self.path)
@@ -246,6 +270,35 @@ def mote_moe_forward_host(layer: MoteLayer, x_host: torch.Tensor, out_host: torc
     _check(lib.mote_moe_forward_host(C.byref(s), _ptr(x_host), _ptr(residual_host), T, _ptr(out_host), _ptr(ws),
                                      ws.numel(), _stream()), "mote_moe_forward_host")
     return out_host
+
+
+class MoteStack:
+    """A list of MoteLayer run back to back with the residual between layers (mote_stack_forward)."""
+
+    def __init__(self, layers):
+        self.layers = list(layers)
+        self._structs = (mote_layer_t * len(self.layers))(*[l.struct() for l in self.layers])
+        self._ws = None
+
+    def workspace(self, T: int) -> torch.Tensor:
+        need = lib.mote_stack_workspace_bytes(self._structs, len(self.layers), T)
+        if need == 0:
+            raise MoteError(2, "mote_stack_workspace_bytes")
+        if self._ws is None or self._ws.numel() < need:
+            self._ws = torch.empty(need, dtype=torch.uint8, device=self.layers[0].tensors["Wr"].device)
+        return self._ws
+
+
+def mote_stack_forward(stack: MoteStack, x: torch.Tensor, out=None, layer_inputs=None):
+    """x[T, d] bf16 -> x_L[T, d] bf16 after all layers; layer_inputs ([L, T, d] bf16) receives every layer's input."""
+    _need_cuda(x, out, layer_inputs)
+    T = x.shape[0]
+    if out is None:
+        out = torch.empty_like(x)
+    ws = stack.workspace(T)
+    _check(lib.mote_stack_forward(stack._structs, len(stack.layers), _ptr(x), T, _ptr(out), _ptr(layer_inputs), _ptr(ws),
+                                  ws.numel(), _stream()), "mote_stack_forward")
+    return out
 
 
 STAGE_NAMES = ["route", "dispatch", "quant_x", "gateup_ternary", "quant_h", "down_ternary", "shared_gateup",

@@ -339,6 +339,49 @@ extern "C" mote_status_t mote_moe_forward(const mote_layer_t* L, const void* x, 
   return MOTE_OK;
 }
 
+extern "C" size_t mote_stack_workspace_bytes(const mote_layer_t* layers, int n_layers, int64_t T_max) {
+  if (!layers || n_layers < 1 || T_max < 0) return 0;
+  size_t core = 0;
+  for (int l = 0; l < n_layers; ++l) {
+    const size_t b = mote_workspace_bytes(layers[l].d, layers[l].f, layers[l].E, layers[l].k, T_max);
+    if (b == 0 || layers[l].d != layers[0].d) return 0;
+    core = std::max(core, b);
+  }
+  return core + 2 * round_up(size_t(T_max) * layers[0].d * 2, 256);
+}
+
+extern "C" mote_status_t mote_stack_forward(const mote_layer_t* layers, int n_layers, const void* x, int64_t T,
+                                            void* out, void* layer_inputs, void* ws, size_t ws_bytes, void* stream_) {
+  if (!layers) return MOTE_ERR_NULL;
+  if (n_layers < 1 || T < 0) return MOTE_ERR_SHAPE;
+  if (T == 0) return MOTE_OK;
+  if (!x || !out || !ws) return MOTE_ERR_NULL;
+  if (x == out) return MOTE_ERR_SHAPE;
+  const size_t need = mote_stack_workspace_bytes(layers, n_layers, T);
+  if (need == 0) return MOTE_ERR_SHAPE;
+  if (ws_bytes < need) return MOTE_ERR_WORKSPACE;
+  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+  const int d = layers[0].d;
+  const size_t row_bytes = size_t(T) * d * 2;
+  const size_t slab = round_up(row_bytes, 256);
+  const size_t core = need - 2 * slab;
+  char* ping = static_cast<char*>(ws) + core;
+  int launches = 0;
+  const void* in = x;
+  for (int l = 0; l < n_layers; ++l) {
+    void* dst = (l == n_layers - 1) ? out : static_cast<void*>(ping + size_t(l & 1) * slab);
+    if (layer_inputs)
+      MOTE_CUDA_OK(cudaMemcpyAsync(static_cast<char*>(layer_inputs) + size_t(l) * row_bytes, in, row_bytes,
+                                   cudaMemcpyDeviceToDevice, stream));
+    const mote_status_t st = mote_moe_forward(&layers[l], in, in, T, dst, nullptr, ws, core, stream);
+    if (st) return st;
+    launches += g_launch_count;
+    in = dst;
+  }
+  g_launch_count = launches;
+  return MOTE_OK;
+}
+
 extern "C" mote_status_t mote_moe_forward_host(const mote_layer_t* L, const void* x_host, const void* residual_host,
                                                int64_t T, void* out_host, void* ws, size_t ws_bytes, void* stream_) {
   if (!L) return MOTE_ERR_NULL;

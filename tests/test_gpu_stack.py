@@ -1,0 +1,78 @@
+"""mote_stack_forward: layers chained with the residual between them (the c5 workload's shape of
+use).  Each layer is checked against the oracle ON THE GPU'S OWN LAYER INPUT (a bf16 rounding
+difference upstream may legitimately flip a routing decision downstream, so parity is per layer),
+and the chain must equal the same layers called one by one, bit for bit."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import mote_oracle as O
+from workloads import synth
+from parity_utils import REL_FRO_TOL, bf16_bits, bf16_tensor
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def mote():
+    import paper_2506_14435_b200 as m
+    return m
+
+
+@pytest.mark.parametrize("T", [1, 40, 150])          # decode path (1, 40) and tensor-core path (150)
+def test_small_stack_per_layer_parity(mote, T):
+    n_layers = 5
+    wl = synth.custom("stack", 128, 256, 4, 2, T, 4100, n_layers=n_layers, w_std=0.08)
+    masters = [synth.master_layer(wl, layer=l) for l in range(n_layers)]
+    layers = [mote.MoteLayer.from_master(m) for m in masters]
+    stack = mote.MoteStack(layers)
+    x_bits = synth.tokens(wl)
+    x = bf16_tensor(x_bits)
+    taps = torch.zeros((n_layers, T, wl.d), dtype=torch.bfloat16, device="cuda")
+    out = mote.mote_stack_forward(stack, x, layer_inputs=taps)
+    torch.cuda.synchronize()
+    assert torch.equal(taps[0], x)
+    # the chain equals layer-by-layer calls
+    cur = x
+    for l, layer in enumerate(layers):
+        assert torch.equal(taps[l], cur)
+        cur = mote.mote_moe_forward(layer, cur, residual=cur)
+    assert torch.equal(cur, out)
+    # every layer against the oracle, on the GPU's input of that layer
+    for l in range(n_layers):
+        layer_or = O.build_layer(masters[l])
+        xin = bf16_bits(taps[l])
+        got_t = taps[l + 1] if l + 1 < n_layers else out
+        idx_taps = layers[l].alloc_taps(T, names=["topk_idx"])
+        mote.mote_moe_forward(layers[l], taps[l].contiguous(), residual=taps[l].contiguous(), taps=idx_taps)
+        ref = O.moe_forward(layer_or, xin, residual_bf16=xin, near_tie_choice=idx_taps["topk_idx"].cpu().numpy())
+        got = O.bf16_to_f32(bf16_bits(got_t)).astype(np.float64)
+        err = np.linalg.norm(got - ref["out"]) / np.linalg.norm(ref["out"])
+        assert err <= REL_FRO_TOL, (l, err)
+
+
+def test_c5_shape_stack_matches_layer_by_layer(mote):
+    wl = synth.WORKLOADS["c5"]
+    layers = [mote.MoteLayer.from_device_draws(wl.d, wl.f, wl.E, wl.k, wl.norm_topk, synth.device_draw(wl, l, "cuda"))
+              for l in range(2)]
+    stack = mote.MoteStack(layers)
+    for T in (1, 32, 300):
+        x = synth.device_tokens(wl, "cuda", T=T)
+        out = mote.mote_stack_forward(stack, x)
+        cur = x
+        for layer in layers:
+            cur = mote.mote_moe_forward(layer, cur, residual=cur)
+        assert torch.equal(cur, out)
+        assert torch.isfinite(out.float()).all()
+
+
+def test_stack_argument_errors(mote):
+    import ctypes as C
+    from paper_2506_14435_b200.binding import mote_layer_t
+    lib = mote.lib
+    arr = (mote_layer_t * 2)(mote_layer_t(128, 256, 4, 2, 1, 0), mote_layer_t(256, 256, 4, 2, 1, 0))
+    assert lib.mote_stack_workspace_bytes(arr, 2, 8) == 0            # layers of different d
+    fake = C.c_void_p(0x1000)
+    assert lib.mote_stack_forward(arr, 0, fake, 4, C.c_void_p(0x2000), None, fake, 1 << 20, None) == 2
+    assert lib.mote_stack_forward(None, 1, fake, 4, C.c_void_p(0x2000), None, fake, 1 << 20, None) == 1
+    assert lib.mote_stack_forward(arr, 1, fake, 4, fake, None, fake, 1 << 20, None) == 2    # out aliases x

@@ -144,3 +144,50 @@ def sample_tokens(offsets: np.ndarray, inv: np.ndarray, k: int, T: int, n_random
     if n_random > 0:
         toks.update(int(t) for t in rng.choice(T, size=min(n_random, T), replace=False))
     return np.array(sorted(toks), dtype=np.int64)
+
+
+def device_draw(wl: Workload, layer: int, device):
+    """Returns draw(name, expert) producing the tensors of one layer directly on `device`, for
+    layer stacks that would take minutes to draw on the host (c5: 36 layers of 0.8 G weights).
+    Same distributions and seeding scheme as the host generators but a different random stream,
+    so these tensors are for timing and for GPU-against-GPU consistency checks, never for the oracle.
+    name: "gate" | "up" | "down" (fp32 [f,d] / [d,f]), "sh_gate" | "sh_up" | "sh_down" (bf16),
+    "Wr" (fp32 [E,d], bf16-representable), "bias" (fp32 [E] or None)."""
+    ids = dict(gate=MAT_GATE, up=MAT_UP, down=MAT_DOWN, sh_gate=MAT_SH_GATE, sh_up=MAT_SH_UP, sh_down=MAT_SH_DOWN,
+               Wr=MAT_ROUTER, bias=MAT_BIAS)
+
+    def gen(expert, mat):
+        g = torch.Generator(device=device)
+        g.manual_seed(((wl.seed * 1009 + layer) * 1009 + expert) * 1009 + mat)
+        return g
+
+    def draw(name: str, expert: int = 0):
+        mat = ids[name]
+        if name == "Wr":
+            w = torch.randn((wl.E, wl.d), generator=gen(0, mat), device=device, dtype=torch.float32) * wl.w_std
+            return w.to(torch.bfloat16).to(torch.float32)
+        if name == "bias":
+            if wl.bias == "zipf":
+                p = torch.arange(1, wl.E + 1, dtype=torch.float64) ** -1.1
+                return torch.log(p / p.sum()).to(torch.float32).to(device)
+            if wl.bias == "normal":
+                return torch.randn((wl.E,), generator=gen(0, mat), device=device, dtype=torch.float32) * 0.5
+            return None
+        shape = (wl.d, wl.f) if name in ("down", "sh_down") else (wl.f, wl.d)
+        w = torch.randn(shape, generator=gen(expert, mat), device=device, dtype=torch.float32) * wl.w_std
+        return w.to(torch.bfloat16) if name.startswith("sh_") else w
+
+    return draw
+
+
+def device_tokens(wl: Workload, device, T: int | None = None, stream: int = 0) -> torch.Tensor:
+    """x[T, d] bf16 drawn on the device (N(0,1), optional outlier channels); see device_draw."""
+    T = wl.T if T is None else T
+    g = torch.Generator(device=device)
+    g.manual_seed(((wl.seed * 1009) * 1009 + stream) * 1009 + MAT_X)
+    x = torch.randn((T, wl.d), generator=g, device=device, dtype=torch.float32)
+    n_out = int(round(wl.outlier_frac * wl.d))
+    if n_out > 0:
+        chans = torch.randperm(wl.d, generator=g, device=device)[:n_out]
+        x[:, chans] *= wl.outlier_gain
+    return x.to(torch.bfloat16)
