@@ -222,7 +222,8 @@ def run_ours(args):
     cur = x
     for layer in layers:
         taps = layer.alloc_taps(wl.T, names=["offsets"])
-        nxt = mote.mote_moe_forward(layer, cur, residual=cur if is_stack else None, taps=taps)
+        nxt = mote.mote_moe_forward(layer, mote.mote_rms_norm(cur) if is_stack else cur,
+                                    residual=cur if is_stack else None, taps=taps)
         touched.append(int((taps["offsets"][1:] - taps["offsets"][:-1] > 0).sum().item()))
         cur = nxt
     experts_touched = sum(touched) / len(touched)
@@ -248,7 +249,8 @@ def run_ours(args):
         tot = {}
         for layer in layers:
             nxt = torch.empty_like(cur)
-            ms = mote_moe_forward_profile(layer, cur, out=nxt, residual=cur if is_stack else None)
+            ms = mote_moe_forward_profile(layer, mote.mote_rms_norm(cur) if is_stack else cur, out=nxt,
+                                          residual=cur if is_stack else None)
             for k_, v in ms.items():
                 tot[k_] = tot.get(k_, 0.0) + v
             cur = nxt
@@ -298,6 +300,8 @@ def run_ours(args):
     roof["peak_source"] = ("of measured" if peaks["source"] == "measured" else "of fallback") + \
         (" (bf16 burst x2 nominal int8:bf16 ratio)" if kind == "int8" else "")
     weight_bytes = len(layers) * (experts_touched * 3 * wl.d * wl.f / 4 + 6.0 * wl.d * wl.f)
+    if not bool(torch.isfinite(out.float()).all()):
+        raise SystemExit("non-finite layer output: the timing would not be valid")
     line = {
         "metric": "MoTE layer tokens/sec (prefill)" if not decode else "MoTE layer tokens/sec (decode batch)",
         "value": tokens_per_s, "unit": "tokens/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
@@ -306,6 +310,7 @@ def run_ours(args):
         "scaling": "weak", "vs_baseline": None, "dtype": "int8xint2->int32 routed, bf16 shared", "data": "synthetic",
         "config": {"workload": wl.name, "d": wl.d, "f": wl.f, "E": wl.E, "k": wl.k, "T_per_gpu": wl.T,
                    "layers": len(layers), "experts_touched_per_layer": experts_touched,
+                   "pre_norm": "rms, eps 1e-6, unit gain" if is_stack else "none (the caller's)",
                    "l2": "flushed between timed iterations (512 MiB write)", "parallelism": f"replicas x{world}"},
         "stage_ms": stage_ms, "roofline": roof,
         "weights_touched_gbs": weight_bytes / (ms_per_step * 1e-3) / 1e9,

@@ -203,24 +203,35 @@ mote_status_t mote_moe_forward_host(const mote_layer_t* L, const void* x_host,
                                     void* ws, size_t ws_bytes, void* stream);
 
 /* ------------------------------------------------------------------------------------------------
- * mote_stack_forward -- n_layers MoTE FFN layers back to back with the residual of Eq. 1-2 between
- * them (attention and the norms of a transformer block are the caller's and are not part of this):
+ * mote_rms_norm -- the LN of Eq. 2 for callers that chain layers: RMS normalisation (as in the
+ * Qwen2.5 models the paper up-cycles), unit gain:
+ *     y[t, :] = bf16( x[t, :] * rsqrt( mean_j x[t, j]^2 + eps ) )        fp32 arithmetic
+ * x_bf16, y_bf16: [T, d] bf16 contiguous, 16-B aligned; y may alias x.  Errors: d % 8 != 0 -> ERR_SHAPE.
+ */
+mote_status_t mote_rms_norm(const void* x_bf16, int64_t T, int64_t d, float eps, void* y_bf16, void* stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * mote_stack_forward -- n_layers MoTE FFN layers back to back as Eq. 1-2 chain them (the attention
+ * sub-block of a transformer layer is not part of this):
  *
- *     x_l = bf16( x_{l-1} + FFN_l(x_{l-1}) + MoE_l(x_{l-1}) ),   l = 1 .. n_layers,  x_0 = x
+ *     x_l = bf16( x_{l-1} + FFN_l(n_l) + MoE_l(n_l) ),  n_l = LN(x_{l-1}),   l = 1 .. n_layers,  x_0 = x
  *
- * i.e. mote_moe_forward(layer l, x_{l-1}, residual = x_{l-1}) chained on one stream, nothing
- * synchronises in between.
+ * LN is mote_rms_norm with rms_eps when rms_eps > 0, and the identity when rms_eps == 0.  Each step
+ * is mote_moe_forward(layer l, n_l, residual = x_{l-1}); everything is chained on one stream and
+ * nothing synchronises in between.
  *
  *   layers_host        in   HOST array of n_layers layer descriptions; all layers share d, f may differ
  *   x_bf16             in   [T, d] bf16 device
  *   out_bf16           out  [T, d] bf16 device = x_{n_layers}; must not alias x_bf16
- *   layer_inputs_bf16  out  NULL, or [n_layers, T, d] bf16 device: x_{l-1} for every layer l (parity tap)
+ *   layer_inputs_bf16  out  NULL, or [n_layers, T, d] bf16 device: the residual stream x_{l-1} entering
+ *                           every layer l (parity tap; n_l follows from it with mote_rms_norm)
  *   ws, ws_bytes            >= mote_stack_workspace_bytes(...), 256-B aligned
- * Errors: as mote_moe_forward; n_layers < 1 or layers of different d -> ERR_SHAPE.
+ * Errors: as mote_moe_forward; n_layers < 1, layers of different d or rms_eps < 0 -> ERR_SHAPE.
  */
 size_t mote_stack_workspace_bytes(const mote_layer_t* layers_host, int n_layers, int64_t T_max);
-mote_status_t mote_stack_forward(const mote_layer_t* layers_host, int n_layers, const void* x_bf16, int64_t T,
-                                 void* out_bf16, void* layer_inputs_bf16, void* ws, size_t ws_bytes, void* stream);
+mote_status_t mote_stack_forward(const mote_layer_t* layers_host, int n_layers, float rms_eps, const void* x_bf16,
+                                 int64_t T, void* out_bf16, void* layer_inputs_bf16, void* ws, size_t ws_bytes,
+                                 void* stream);
 
 /* mote_moe_forward with a CUDA event recorded on `stream` between the stages; waits for the stream
  * and writes the device time of each stage, in milliseconds, to stage_ms_host[MOTE_N_STAGES]:

@@ -290,6 +290,18 @@ def shared_ffn(x_bf16, Wg_bf16, Wu_bf16, Wd_bf16) -> np.ndarray:
 
 
 # --------------------------------------------------------------------------------------------
+# Eq. 1-2  LN in front of the layer: RMS normalisation with unit gain (Qwen2.5's norm)
+# --------------------------------------------------------------------------------------------
+
+
+def rms_norm(x_bf16: np.ndarray, eps: float) -> np.ndarray:
+    """LN(x) of Eq. 2 as the Qwen2.5 backbone applies it: x / sqrt(mean(x^2) + eps) per token,
+    no mean subtraction, unit gain; fp64 on the bf16 values, not rounded."""
+    x = bf16_to_f32(x_bf16).astype(np.float64)
+    return x / np.sqrt(np.mean(x * x, axis=1, keepdims=True) + eps)
+
+
+# --------------------------------------------------------------------------------------------
 # Eq. 2, 4  the whole layer
 # --------------------------------------------------------------------------------------------
 

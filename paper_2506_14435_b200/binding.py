@@ -61,8 +61,10 @@ lib.mote_moe_forward.argtypes = [C.POINTER(mote_layer_t), C.c_void_p, C.c_void_p
 lib.mote_stack_workspace_bytes.restype = C.c_size_t
 lib.mote_stack_workspace_bytes.argtypes = [C.POINTER(mote_layer_t), C.c_int, C.c_int64]
 lib.mote_stack_forward.restype = C.c_int
-lib.mote_stack_forward.argtypes = [C.POINTER(mote_layer_t), C.c_int, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p,
-                                   C.c_void_p, C.c_size_t, C.c_void_p]
+lib.mote_stack_forward.argtypes = [C.POINTER(mote_layer_t), C.c_int, C.c_float, C.c_void_p, C.c_int64, C.c_void_p,
+                                   C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+lib.mote_rms_norm.restype = C.c_int
+lib.mote_rms_norm.argtypes = [C.c_void_p, C.c_int64, C.c_int64, C.c_float, C.c_void_p, C.c_void_p]
 lib.mote_moe_forward_host.restype = C.c_int
 lib.mote_moe_forward_host.argtypes = [C.POINTER(mote_layer_t), C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p,
                                       C.c_void_p, C.c_size_t, C.c_void_p]
@@ -289,15 +291,26 @@ class MoteStack:
         return self._ws
 
 
-def mote_stack_forward(stack: MoteStack, x: torch.Tensor, out=None, layer_inputs=None):
-    """x[T, d] bf16 -> x_L[T, d] bf16 after all layers; layer_inputs ([L, T, d] bf16) receives every layer's input."""
+def mote_rms_norm(x: torch.Tensor, eps: float = 1e-6, out=None):
+    """The LN of Eq. 2 (RMS normalisation, unit gain) of x[T, d] bf16."""
+    _need_cuda(x, out)
+    if out is None:
+        out = torch.empty_like(x)
+    _check(lib.mote_rms_norm(_ptr(x), x.shape[0], x.shape[1], eps, _ptr(out), _stream()), "mote_rms_norm")
+    return out
+
+
+def mote_stack_forward(stack: MoteStack, x: torch.Tensor, out=None, layer_inputs=None, rms_eps: float = 1e-6):
+    """x[T, d] bf16 -> x_L[T, d] bf16 after all layers (Eq. 1-2 chained, LN = RMS norm; rms_eps = 0
+    chains the layers without normalisation); layer_inputs ([L, T, d] bf16) receives the residual
+    stream entering every layer."""
     _need_cuda(x, out, layer_inputs)
     T = x.shape[0]
     if out is None:
         out = torch.empty_like(x)
     ws = stack.workspace(T)
-    _check(lib.mote_stack_forward(stack._structs, len(stack.layers), _ptr(x), T, _ptr(out), _ptr(layer_inputs), _ptr(ws),
-                                  ws.numel(), _stream()), "mote_stack_forward")
+    _check(lib.mote_stack_forward(stack._structs, len(stack.layers), rms_eps, _ptr(x), T, _ptr(out), _ptr(layer_inputs),
+                                  _ptr(ws), ws.numel(), _stream()), "mote_stack_forward")
     return out
 
 

@@ -347,13 +347,14 @@ extern "C" size_t mote_stack_workspace_bytes(const mote_layer_t* layers, int n_l
     if (b == 0 || layers[l].d != layers[0].d) return 0;
     core = std::max(core, b);
   }
-  return core + 2 * round_up(size_t(T_max) * layers[0].d * 2, 256);
+  return core + 3 * round_up(size_t(T_max) * layers[0].d * 2, 256);   // two residual-stream slabs + LN output
 }
 
-extern "C" mote_status_t mote_stack_forward(const mote_layer_t* layers, int n_layers, const void* x, int64_t T,
-                                            void* out, void* layer_inputs, void* ws, size_t ws_bytes, void* stream_) {
+extern "C" mote_status_t mote_stack_forward(const mote_layer_t* layers, int n_layers, float rms_eps, const void* x,
+                                            int64_t T, void* out, void* layer_inputs, void* ws, size_t ws_bytes,
+                                            void* stream_) {
   if (!layers) return MOTE_ERR_NULL;
-  if (n_layers < 1 || T < 0) return MOTE_ERR_SHAPE;
+  if (n_layers < 1 || T < 0 || !(rms_eps >= 0.0f)) return MOTE_ERR_SHAPE;
   if (T == 0) return MOTE_OK;
   if (!x || !out || !ws) return MOTE_ERR_NULL;
   if (x == out) return MOTE_ERR_SHAPE;
@@ -364,19 +365,28 @@ extern "C" mote_status_t mote_stack_forward(const mote_layer_t* layers, int n_la
   const int d = layers[0].d;
   const size_t row_bytes = size_t(T) * d * 2;
   const size_t slab = round_up(row_bytes, 256);
-  const size_t core = need - 2 * slab;
+  const size_t core = need - 3 * slab;
   char* ping = static_cast<char*>(ws) + core;
+  void* normed = ping + 2 * slab;
   int launches = 0;
-  const void* in = x;
+  const void* res = x;                                 // residual stream x_{l-1}
   for (int l = 0; l < n_layers; ++l) {
     void* dst = (l == n_layers - 1) ? out : static_cast<void*>(ping + size_t(l & 1) * slab);
     if (layer_inputs)
-      MOTE_CUDA_OK(cudaMemcpyAsync(static_cast<char*>(layer_inputs) + size_t(l) * row_bytes, in, row_bytes,
+      MOTE_CUDA_OK(cudaMemcpyAsync(static_cast<char*>(layer_inputs) + size_t(l) * row_bytes, res, row_bytes,
                                    cudaMemcpyDeviceToDevice, stream));
-    const mote_status_t st = mote_moe_forward(&layers[l], in, in, T, dst, nullptr, ws, core, stream);
+    const void* in = res;
+    if (rms_eps > 0.0f) {
+      g_launch_count = 0;
+      const mote_status_t sn = launch_rms_norm(res, T, d, rms_eps, normed, stream);
+      if (sn) return sn;
+      launches += g_launch_count;
+      in = normed;
+    }
+    const mote_status_t st = mote_moe_forward(&layers[l], in, res, T, dst, nullptr, ws, core, stream);
     if (st) return st;
     launches += g_launch_count;
-    in = dst;
+    res = dst;
   }
   g_launch_count = launches;
   return MOTE_OK;

@@ -101,6 +101,9 @@ bool decode_stream_supported(int d, int f, int E, int k, int64_t T);
 // phase 0: prologue, 1: gate/up (routed + shared), 2: down (routed + shared); Q_a(h) runs between 1 and 2
 mote_status_t launch_decode_stream(const DecodeStreamArgs& a, int phase, cudaStream_t stream);
 
+// y = bf16(x * rsqrt(mean(x^2) + eps)) per row (the LN of Eq. 2, unit gain)
+mote_status_t launch_rms_norm(const void* x, int64_t T, int d, float eps, void* y, cudaStream_t stream);
+
 // out = [residual +] s + sum_j w_j * y[perm[t*k+j]]
 mote_status_t launch_combine(const float* s, const float* y, const float* w, const int32_t* perm,
                              const void* residual, int64_t T, int d, int k, void* out_bf16,

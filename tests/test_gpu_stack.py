@@ -19,8 +19,23 @@ def mote():
     return m
 
 
+@pytest.mark.parametrize("T,d", [(1, 64), (5, 896), (33, 2048), (300, 256), (3, 8192)])
+def test_rms_norm(mote, T, d):
+    rng = np.random.default_rng(T * 31 + d)
+    x = O.f32_to_bf16_rn((rng.standard_normal((T, d)) * rng.uniform(0.01, 40.0, size=(T, 1))).astype(np.float32))
+    if T > 2:
+        x[1] = 0
+    want = O.rms_norm(x, 1e-6)
+    got = O.bf16_to_f32(bf16_bits(mote.mote_rms_norm(bf16_tensor(x), 1e-6))).astype(np.float64)
+    # fp32 arithmetic and one bf16 rounding: within one bf16 ulp (2^-8 relative) of the fp64 value
+    assert np.all(np.abs(got - want) <= np.abs(want) * 2.0 ** -8 + 1e-30)
+    err = np.linalg.norm(got - want) / max(np.linalg.norm(want), 1e-30)
+    assert err <= REL_FRO_TOL
+
+
+@pytest.mark.parametrize("rms_eps", [1e-6, 0.0])
 @pytest.mark.parametrize("T", [1, 40, 150])          # decode path (1, 40) and tensor-core path (150)
-def test_small_stack_per_layer_parity(mote, T):
+def test_small_stack_per_layer_parity(mote, T, rms_eps):
     n_layers = 5
     wl = synth.custom("stack", 128, 256, 4, 2, T, 4100, n_layers=n_layers, w_std=0.08)
     masters = [synth.master_layer(wl, layer=l) for l in range(n_layers)]
@@ -29,23 +44,26 @@ def test_small_stack_per_layer_parity(mote, T):
     x_bits = synth.tokens(wl)
     x = bf16_tensor(x_bits)
     taps = torch.zeros((n_layers, T, wl.d), dtype=torch.bfloat16, device="cuda")
-    out = mote.mote_stack_forward(stack, x, layer_inputs=taps)
+    out = mote.mote_stack_forward(stack, x, layer_inputs=taps, rms_eps=rms_eps)
     torch.cuda.synchronize()
     assert torch.equal(taps[0], x)
+    norm = (lambda t: mote.mote_rms_norm(t.contiguous(), rms_eps)) if rms_eps > 0 else (lambda t: t.contiguous())
     # the chain equals layer-by-layer calls
     cur = x
     for l, layer in enumerate(layers):
         assert torch.equal(taps[l], cur)
-        cur = mote.mote_moe_forward(layer, cur, residual=cur)
+        cur = mote.mote_moe_forward(layer, norm(cur), residual=cur)
     assert torch.equal(cur, out)
-    # every layer against the oracle, on the GPU's input of that layer
+    # every layer against the oracle, on the GPU's own input and residual of that layer
     for l in range(n_layers):
         layer_or = O.build_layer(masters[l])
-        xin = bf16_bits(taps[l])
+        res = taps[l].contiguous()
+        xin_t = norm(res)
         got_t = taps[l + 1] if l + 1 < n_layers else out
         idx_taps = layers[l].alloc_taps(T, names=["topk_idx"])
-        mote.mote_moe_forward(layers[l], taps[l].contiguous(), residual=taps[l].contiguous(), taps=idx_taps)
-        ref = O.moe_forward(layer_or, xin, residual_bf16=xin, near_tie_choice=idx_taps["topk_idx"].cpu().numpy())
+        mote.mote_moe_forward(layers[l], xin_t, residual=res, taps=idx_taps)
+        ref = O.moe_forward(layer_or, bf16_bits(xin_t), residual_bf16=bf16_bits(res),
+                            near_tie_choice=idx_taps["topk_idx"].cpu().numpy())
         got = O.bf16_to_f32(bf16_bits(got_t)).astype(np.float64)
         err = np.linalg.norm(got - ref["out"]) / np.linalg.norm(ref["out"])
         assert err <= REL_FRO_TOL, (l, err)
@@ -61,7 +79,7 @@ def test_c5_shape_stack_matches_layer_by_layer(mote):
         out = mote.mote_stack_forward(stack, x)
         cur = x
         for layer in layers:
-            cur = mote.mote_moe_forward(layer, cur, residual=cur)
+            cur = mote.mote_moe_forward(layer, mote.mote_rms_norm(cur, 1e-6), residual=cur)
         assert torch.equal(cur, out)
         assert torch.isfinite(out.float()).all()
 
@@ -73,6 +91,9 @@ def test_stack_argument_errors(mote):
     arr = (mote_layer_t * 2)(mote_layer_t(128, 256, 4, 2, 1, 0), mote_layer_t(256, 256, 4, 2, 1, 0))
     assert lib.mote_stack_workspace_bytes(arr, 2, 8) == 0            # layers of different d
     fake = C.c_void_p(0x1000)
-    assert lib.mote_stack_forward(arr, 0, fake, 4, C.c_void_p(0x2000), None, fake, 1 << 20, None) == 2
-    assert lib.mote_stack_forward(None, 1, fake, 4, C.c_void_p(0x2000), None, fake, 1 << 20, None) == 1
-    assert lib.mote_stack_forward(arr, 1, fake, 4, fake, None, fake, 1 << 20, None) == 2    # out aliases x
+    eps = C.c_float(1e-6)
+    assert lib.mote_stack_forward(arr, 0, eps, fake, 4, C.c_void_p(0x2000), None, fake, 1 << 20, None) == 2
+    assert lib.mote_stack_forward(None, 1, eps, fake, 4, C.c_void_p(0x2000), None, fake, 1 << 20, None) == 1
+    assert lib.mote_stack_forward(arr, 1, eps, fake, 4, fake, None, fake, 1 << 20, None) == 2    # out aliases x
+    assert lib.mote_stack_forward(arr, 1, C.c_float(-1.0), fake, 4, C.c_void_p(0x2000), None, fake, 1 << 20, None) == 2
+    assert lib.mote_rms_norm(fake, 4, 12, eps, fake, None) == 2 and lib.mote_rms_norm(None, 4, 16, eps, fake, None) == 1

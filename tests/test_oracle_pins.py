@@ -256,3 +256,23 @@ def test_dispatch_is_a_stable_counting_sort():
     for e in range(E):
         assert offsets[e + 1] - offsets[e] == int((idx == e).sum())
     assert offsets[4] == offsets[3]
+
+
+# ------------------------------------------------------------------ LN of Eq. 2 (RMS norm)
+def test_rms_norm_against_library_and_invariants():
+    rng = np.random.default_rng(21)
+    x = O.f32_to_bf16_rn((rng.standard_normal((7, 96)) * np.array([[0.01], [1], [30], [1], [2], [5], [0.5]])).astype(np.float32))
+    got = O.rms_norm(x, 1e-6)
+    xt = torch.from_numpy(O.bf16_to_f32(x).astype(np.float64))
+    want = torch.nn.functional.rms_norm(xt, (96,), eps=1e-6).numpy()          # library routine, fp64
+    assert np.allclose(got, want, rtol=1e-12, atol=0)
+    assert np.allclose(np.sqrt(np.mean(got * got, axis=1))[1:], 1.0, atol=1e-5)   # unit rms (eps negligible)
+    # scale invariance for power-of-two scalings (exact in bf16), eps -> 0
+    x4 = O.f32_to_bf16_rn(O.bf16_to_f32(x) * np.float32(4.0))
+    assert np.allclose(O.rms_norm(x4, 0.0), O.rms_norm(x, 0.0), rtol=1e-12)
+    # a one-hot row of height a normalises to sqrt(d) at that position
+    one = np.zeros((1, 64), np.float32); one[0, 5] = -3.0
+    r = O.rms_norm(O.f32_to_bf16_rn(one), 0.0)
+    assert abs(r[0, 5] + 8.0) < 1e-12 and np.count_nonzero(r) == 1
+    # all-zero row stays zero when eps > 0
+    assert np.all(O.rms_norm(np.zeros((1, 16), np.uint16), 1e-6) == 0)
