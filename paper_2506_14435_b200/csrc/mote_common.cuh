@@ -135,20 +135,22 @@ __device__ __forceinline__ float glu_h(int acc_g, int acc_u, float c_g, float c_
 //   s'  = fl(g * rcp.approx(den'))  (rcp: <= 2^-23, product 2^-24) vs s = fl(g / den) -> <= 1.0e-6
 //   h'  = fl(u * s')                                             vs h  -> <= 1.12e-6 < 19 ulp
 // bf16_rn(h') == bf16_rn(h) unless h' lies within 19 fp32 ulps of the midpoint between two bf16
-// values; the flag is raised within 64 ulps of a midpoint (low 16 bits in [0x7FC0, 0x8040]), and
+// values; the flag is raised within 32 ulps of a midpoint (low 16 bits in [0x7FE0, 0x8020]), and
 // for |t| > 64 where the clamp, overflow or gradual underflow could make the two differ more.
-// Flagged elements (about 0.2 %) are recomputed with glu_h.  The caller must also send rows with
+// Flagged elements (about 0.1 %) are recomputed with glu_h.  The caller must also send rows with
 // c_g * c_u <= 1e-12 to glu_h (h' could be subnormal there).
 __device__ __forceinline__ float glu_h_fast(int acc_g, int acc_u, float c_g, float c_u, bool& redo) {
   const float g = __fmul_rn(i2f_small(acc_g), c_g);
   const float u = __fmul_rn(i2f_small(acc_u), c_u);
   const float t = __fmul_rn(-g, 1.4426950408889634f);
   float e, rc;
-  asm("ex2.approx.f32 %0, %1;" : "=f"(e) : "f"(t));
+  // .ftz: single instructions; with |t| <= 64 neither the operands nor the results are subnormal
+  // (a subnormal t is flushed to 0, where 2^t = 1 to well within the error budget)
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(t));
   const float den = __fadd_rn(1.0f, e);
-  asm("rcp.approx.f32 %0, %1;" : "=f"(rc) : "f"(den));
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(rc) : "f"(den));
   const float h = __fmul_rn(u, __fmul_rn(g, rc));
-  redo = ((__float_as_uint(h) & 0xFFFFu) - 0x7FC0u) <= 0x80u || !(fabsf(t) <= 64.0f);
+  redo = ((__float_as_uint(h) & 0xFFFFu) - 0x7FE0u) <= 0x40u || !(fabsf(t) <= 64.0f);
   return h;
 }
 
@@ -157,6 +159,15 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   uint32_t d;
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
   return d;
+}
+
+// SiLU for the shared (bf16, not bit-pinned) expert: g / (1 + 2^(-g*log2e)) on the special-function unit
+__device__ __forceinline__ float silu_fast(float g) {
+  float e, rc;
+  const float t = fminf(fmaxf(g * -1.4426950408889634f, -80.0f), 80.0f);
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(t));
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(rc) : "f"(1.0f + e));
+  return g * rc;
 }
 
 // scale of one ternary linear output row: alpha * (beta / 127)

@@ -355,7 +355,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
 #pragma unroll
                 for (int j = 0; j < 16; ++j) {
                   const float g = __uint_as_float(rg[j]);
-                  hv[j] = __uint_as_float(ru[j]) * __fdividef(g, 1.0f + __expf(-g));
+                  hv[j] = __uint_as_float(ru[j]) * silu_fast(g);
                 }
               }
               uint32_t packed[8];
