@@ -37,8 +37,9 @@ NOMINAL_INT8_OVER_BF16 = 2.0      # dense tensor peak ratio int8 : bf16 (4.5 vs 
 def parse_workload(name: str) -> synth.Workload:
     if name.startswith("c3-"):
         return synth.WORKLOADS["c3"].with_T(int(name[3:]))
-    if name.startswith("c5-"):
-        return synth.WORKLOADS["c5"].with_T(int(name[3:]))
+    if "-" in name:                                     # stacked workloads: c5-32, p3-1, p05-2048 ...
+        base, T = name.split("-", 1)
+        return synth.WORKLOADS[base].with_T(int(T))
     return synth.WORKLOADS[name]
 
 

@@ -48,3 +48,15 @@ def test_c4_full_size_sampled(mote):
     rep = _sampled_parity(mote, synth.WORKLOADS["c4"], n_random=64, max_boundary_tokens=200)
     assert rep["rel_fro"] < 5e-3
     assert rep["counts"].min() >= 0 and rep["counts"].sum() == 2 * 8192
+
+
+@pytest.mark.parametrize("T", [1, 48, 333])
+def test_paper_configuration_top1_full_softmax_gate(mote, T):
+    # the paper's 0.5B model layer: 1 shared + 4 routed experts, top-1, gate weight = P(x)_i of Eq. 3
+    wl = synth.WORKLOADS["p05"].with_T(T)
+    master = synth.master_layer(wl)
+    layer_or = O.build_layer(master)
+    layer_gpu = mote.MoteLayer.from_master(master)
+    rep = check_forward(mote, layer_gpu, layer_or, synth.tokens(wl))
+    assert rep["rel_fro"] < 5e-3
+    assert rep["counts"].sum() == T

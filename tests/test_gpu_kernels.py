@@ -114,3 +114,28 @@ def test_route_topk_many_experts_and_ties(mote):
             assert list(idx[t]).index(3) < list(idx[t]).index(40)
     ok = ~ref["near_tie"]
     assert np.array_equal(idx[ok], ref["idx"][ok])
+
+
+def test_quant_act_every_bf16_value_under_many_scales(mote):
+    """The kernels evaluate 127*x/beta as x * fl(127 * fl(1/beta)) and divide only near a rounding
+    tie; this must give the oracle's integer for EVERY bf16 x with |x| <= beta.  Each row holds beta
+    and all non-negative (or all non-positive) bf16 values below it."""
+    rng = np.random.default_rng(77)
+    betas = [0x3F80, 0x4040, 0x42FE, 0x3F81, 0x3FFF, 0x3400, 0x4B00, 0x0080, 0x1234, 0x7000]   # bf16 bit patterns
+    betas += [int(b) for b in rng.integers(0x2000, 0x6000, size=50)]
+    rows = []
+    for b in betas:
+        vals = np.arange(0, b + 1, dtype=np.uint32)            # all magnitudes up to beta (bit patterns are ordered)
+        if len(vals) > 32768:
+            vals = np.concatenate([vals[-16384:], rng.choice(vals[:-16384], 16384, replace=False)])
+        for sign in (0, 0x8000):
+            row = np.zeros(32768, np.uint16)
+            row[: len(vals)] = (vals | sign).astype(np.uint16)
+            row[len(vals) - 1 if len(vals) <= 32768 else 0] = b   # beta itself, positive
+            rows.append(row)
+    x = np.stack(rows)
+    q, beta, rowsum = O.quant_act(x)
+    gq, gb, gs = mote.mote_quant_act(bf16_tensor(x))
+    assert np.array_equal(gb.cpu().numpy(), beta)
+    assert np.array_equal(gq.cpu().numpy(), q)
+    assert np.array_equal(gs.cpu().numpy(), rowsum)

@@ -16,6 +16,8 @@ of the public instruction / evaluation sets, which an FFN layer only sees as [T,
   c3  d=1536 f=8960  E=8  k=2  T in {1,8,32,64}          router bias ln p_e, p_e ~ (e+1)^-1.1
   c4  d=2048 f=11008 E=16 k=2  T=8192                    outlier channels, router bias N(0,0.5^2)
   c5  36 layers of c4's shape, T in {1,32,2048}          plain tokens, no bias
+  p05 / p15 / p3  the paper's own MoTE models: E=4, top-1, gate = softmax over all experts,
+      24 / 28 / 36 layers of the Qwen2.5-0.5B / 1.5B / 3B FFN shape, 2048-token sequences
 """
 from __future__ import annotations
 
@@ -53,6 +55,11 @@ WORKLOADS = {
     "c3": Workload("c3", 1536, 8960, 8, 2, 64, 1003, bias="zipf"),
     "c4": Workload("c4", 2048, 11008, 16, 2, 8192, 1004, outlier_frac=0.01, bias="normal"),
     "c5": Workload("c5", 2048, 11008, 16, 2, 2048, 1005, n_layers=36),
+    # the configuration the paper trains and evaluates (Section 4.1, App. B): 1 shared + 4 routed
+    # experts, top-1, the gate weight is P(x)_i of Eq. 3 over all experts; 2048-token sequences
+    "p05": Workload("p05", 896, 4864, 4, 1, 2048, 1011, n_layers=24, norm_topk=0),
+    "p15": Workload("p15", 1536, 8960, 4, 1, 2048, 1012, n_layers=28, norm_topk=0),
+    "p3": Workload("p3", 2048, 11008, 4, 1, 2048, 1013, n_layers=36, norm_topk=0),
 }
 C3_BATCHES = (1, 8, 32, 64)
 C5_BATCHES = (1, 32, 2048)
