@@ -112,6 +112,113 @@ __global__ void __launch_bounds__(kDispatchThreads) dispatch_kernel(const int32_
   }
 }
 
+// ------------------------------------------------------------------------------------------------
+// Block-wise dispatch for long prefills.  The router leaves, for every block of kRouteBlockTokens
+// tokens, the number of its pairs per expert (blk_hist[n_blk][E]).  This kernel turns them into
+//   offsets[E+1]          first sorted row of every expert
+//   blk_base[n_blk][E]    first sorted row of the block's pairs of that expert
+// (experts outermost, blocks in order: the same stable order as above) and writes the tile tables.
+// The rank of a pair inside its block is recomputed by the activation quantizer, which then knows
+// the sorted row of every pair without a pass of its own.  One CTA, one warp per expert: lane l
+// sums a contiguous range of blocks, a shuffle scan orders the ranges, a second walk writes the bases.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kDispatchThreads) dispatch_scan_kernel(const int32_t* __restrict__ blk_hist, int n_blk,
+                                                                         int E, int32_t* __restrict__ offsets,
+                                                                         int32_t* __restrict__ blk_base,
+                                                                         int4* __restrict__ tiles_routed,
+                                                                         int4* __restrict__ tiles_shared, int T) {
+  __shared__ int s_count[MOTE_MAX_EXPERTS];
+  __shared__ int s_first[MOTE_MAX_EXPERTS];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  constexpr int kPer = 16;                             // blocks per lane and chunk: 16 independent loads
+  // totals per expert (two rounds of 32 warps cover MOTE_MAX_EXPERTS = 64)
+#pragma unroll
+  for (int r = 0; r < 2; ++r) {
+    const int e = warp + 32 * r;
+    if (e < E) {
+      int tot = 0;
+      for (int c0 = 0; c0 < n_blk; c0 += 32 * kPer) {
+        int v[kPer];
+#pragma unroll
+        for (int i = 0; i < kPer; ++i) {
+          const int b = c0 + lane * kPer + i;
+          v[i] = b < n_blk ? blk_hist[b * E + e] : 0;
+        }
+#pragma unroll
+        for (int i = 0; i < kPer; ++i) tot += v[i];
+      }
+      tot = warp_sum(tot);
+      if (lane == 0) s_count[e] = tot;
+    }
+  }
+  __syncthreads();
+  if (tid == 0) {
+    int run = 0;
+    for (int e = 0; e < E; ++e) {
+      offsets[e] = run;
+      s_first[e] = run;
+      run += s_count[e];
+    }
+    offsets[E] = run;
+  }
+  if (tid == 32 && tiles_routed) {
+    int n = 0, run = 0;
+    for (int e = 0; e < E; ++e) {
+      const int cnt = s_count[e];
+      for (int r = 0; r < cnt; r += 128) tiles_routed[1 + n++] = make_int4(e, run + r, min(128, cnt - r), 0);
+      run += cnt;
+    }
+    tiles_routed[0] = make_int4(n, 0, 0, 0);
+  }
+  if (tiles_shared) {
+    const int n = (T + 127) / 128;
+    for (int i = tid; i < n; i += kDispatchThreads) tiles_shared[1 + i] = make_int4(0, i * 128, min(128, T - i * 128), 0);
+    if (tid == 0) tiles_shared[0] = make_int4(n, 0, 0, 0);
+  }
+  __syncthreads();
+  // bases: blocks in order inside every expert
+#pragma unroll
+  for (int r = 0; r < 2; ++r) {
+    const int e = warp + 32 * r;
+    if (e < E) {
+      int carry = s_first[e];
+      for (int c0 = 0; c0 < n_blk; c0 += 32 * kPer) {
+        int v[kPer];
+        int tot = 0;
+#pragma unroll
+        for (int i = 0; i < kPer; ++i) {
+          const int b = c0 + lane * kPer + i;
+          v[i] = b < n_blk ? blk_hist[b * E + e] : 0;
+          tot += v[i];
+        }
+        int incl = tot;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int n = __shfl_up_sync(0xffffffffu, incl, o);
+          if (lane >= o) incl += n;
+        }
+        int run = carry + incl - tot;
+#pragma unroll
+        for (int i = 0; i < kPer; ++i) {
+          const int b = c0 + lane * kPer + i;
+          if (b < n_blk) blk_base[b * E + e] = run;
+          run += v[i];
+        }
+        carry += __shfl_sync(0xffffffffu, incl, 31);
+      }
+    }
+  }
+}
+
+mote_status_t launch_dispatch_scan(const int32_t* blk_hist, int n_blk, int E, int32_t* offsets, int32_t* blk_base,
+                                   int4* tiles_routed, int4* tiles_shared, int64_t T, cudaStream_t stream) {
+  dispatch_scan_kernel<<<1, kDispatchThreads, 0, stream>>>(blk_hist, n_blk, E, offsets, blk_base, tiles_routed,
+                                                           tiles_shared, (int)T);
+  ++g_launch_count;
+  MOTE_LAUNCH_OK();
+  return MOTE_OK;
+}
+
 mote_status_t launch_dispatch(const int32_t* idx, int64_t P, int E, int32_t* offsets, int32_t* perm,
                               int32_t* inv, int4* tiles_routed, int4* tiles_shared, int64_t T,
                               cudaStream_t stream) {

@@ -25,7 +25,7 @@ static inline void stage_mark(int i, cudaStream_t stream) {
 
 struct Plan {
   size_t status, topk_idx, topk_w, offsets, perm, inv;
-  size_t qx, beta_x, rowsum_x, h, qh, beta_h, rowsum_h, y, hs, s, tiles_routed, tiles_shared;
+  size_t qx, beta_x, rowsum_x, h, qh, beta_h, rowsum_h, y, hs, s, tiles_routed, tiles_shared, blk_hist, blk_base;
   size_t total;
 };
 
@@ -52,6 +52,9 @@ static Plan make_plan(int d, int f, int E, int k, int64_t T) {
   p.s = take(size_t(T) * d * 4);
   p.tiles_routed = take((1 + P / 128 + E) * 16);
   p.tiles_shared = take((1 + (size_t(T) + 127) / 128) * 16);
+  const size_t n_blk = (size_t(T) + kRouteBlockTokens - 1) / kRouteBlockTokens;
+  p.blk_hist = take(n_blk * E * 4);
+  p.blk_base = take(n_blk * E * 4);
   p.total = off;
   return p;
 }
@@ -248,17 +251,28 @@ extern "C" mote_status_t mote_moe_forward(const mote_layer_t* L, const void* x, 
   MOTE_CUDA_OK(cudaMemsetAsync(status, 0, 4, stream));
   stage_mark(0, stream);
   // S1 router, S2 dispatch
-  st = launch_route_topk(x, T, d, L->Wr, L->router_bias, E, k, L->norm_topk, topk_idx, topk_w, nullptr, stream);
+  // block-wise dispatch: the tensor-core router (d % 32 == 0) leaves per-block expert counts, a small
+  // scan turns them into bases, and Q_a(x) derives every pair's sorted row itself
+  const bool blockwise = tensor && (d % 32 == 0);
+  auto* blk_hist = reinterpret_cast<int32_t*>(base + pl.blk_hist);
+  auto* blk_base = reinterpret_cast<int32_t*>(base + pl.blk_base);
+  const int n_blk = (int)((T + kRouteBlockTokens - 1) / kRouteBlockTokens);
+  st = launch_route_topk(x, T, d, L->Wr, L->router_bias, E, k, L->norm_topk, topk_idx, topk_w, nullptr,
+                         blockwise ? blk_hist : nullptr, stream);
   if (st) return st;
   stage_mark(1, stream);
-  st = launch_dispatch(topk_idx, P, E, offsets, perm, inv, tensor ? tiles_routed : nullptr,
-                       tensor ? tiles_shared : nullptr, T, stream);
+  st = blockwise ? launch_dispatch_scan(blk_hist, n_blk, E, offsets, blk_base, tiles_routed, tiles_shared, T, stream)
+                 : launch_dispatch(topk_idx, P, E, offsets, perm, inv, tensor ? tiles_routed : nullptr,
+                                   tensor ? tiles_shared : nullptr, T, stream);
   if (st) return st;
   stage_mark(2, stream);
   // S3 Q_a(x), written once per selected expert into the expert-sorted rows
   QuantActArgs qa{};
   qa.x = x; qa.T = T; qa.d = d; qa.ldx = d; qa.q = qx; qa.beta = beta_x; qa.rowsum = rowsum_x;
   qa.perm = perm; qa.k = k; qa.interleave = interleave;
+  if (blockwise) {
+    qa.topk_idx = topk_idx; qa.blk_base = blk_base; qa.E = E; qa.perm_out = perm; qa.inv_out = inv;
+  }
   st = launch_quant_act(qa, true, stream);
   if (st) return st;
   stage_mark(3, stream);

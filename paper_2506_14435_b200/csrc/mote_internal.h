@@ -16,7 +16,11 @@ struct QuantActArgs {
   int8_t* q;            // [rows, d]
   float* beta;          // [rows]
   int32_t* rowsum;      // [rows] or null
-  const int32_t* perm;  // scatter variant: pair (t*k+j) -> destination row
+  const int32_t* perm;  // scatter variant: pair (t*k+j) -> destination row (when blk_base is null)
+  // scatter variant with the block-wise dispatch: the destination row is derived here from the
+  // top-k indices and the per-block bases, and written to perm_out / inv_out
+  const int32_t* topk_idx; const int32_t* blk_base; int E;
+  int32_t* perm_out; int32_t* inv_out;
   int k;
   int interleave;       // 1: store each unit of 16 codes k-interleaved
   int group;            // threads per row (set by the launcher)
@@ -24,9 +28,12 @@ struct QuantActArgs {
 mote_status_t launch_quant_act(const QuantActArgs& a, bool scatter, cudaStream_t stream);
 
 // Router (Eq. 3).  Arguments as mote_route_topk.
+// blk_hist (optional, written only by the tensor-core kernel, i.e. when d % 32 == 0):
+// [ceil(T / kRouteBlockTokens)][E] pairs per expert of every block of tokens.
+constexpr int kRouteBlockTokens = 16;
 mote_status_t launch_route_topk(const void* x, int64_t T, int d, const float* Wr, const float* bias,
                                 int E, int k, int norm_topk, int32_t* idx, float* w, float* logits,
-                                cudaStream_t stream);
+                                int32_t* blk_hist, cudaStream_t stream);
 
 // Stable grouping of the T*k pairs by expert: offsets[E+1], perm[P] (pair -> row), inv[P] (row -> pair).
 // Optionally also writes the 128-row tile tables of the tensor-core GEMMs ([0] = {count},
@@ -35,6 +42,10 @@ mote_status_t launch_route_topk(const void* x, int64_t T, int d, const float* Wr
 mote_status_t launch_dispatch(const int32_t* idx, int64_t P, int E, int32_t* offsets, int32_t* perm,
                               int32_t* inv, int4* tiles_routed, int4* tiles_shared, int64_t T,
                               cudaStream_t stream);
+
+// Block-wise variant: offsets, per-block bases and the tile tables from the router's block histograms.
+mote_status_t launch_dispatch_scan(const int32_t* blk_hist, int n_blk, int E, int32_t* offsets, int32_t* blk_base,
+                                   int4* tiles_routed, int4* tiles_shared, int64_t T, cudaStream_t stream);
 
 // CUDA-core (dp4a) grouped ternary GEMMs.  qa rows are in expert-sorted order, canonical k order.
 struct TernaryGemmArgs {

@@ -102,7 +102,30 @@ __global__ void __launch_bounds__(256) quant_act_kernel(QuantActArgs a) {
 
   const int n_dst = kScatter ? a.k : 1;
   for (int j = 0; j < n_dst; ++j) {
-    const int64_t dst = kScatter ? int64_t(a.perm[row * a.k + j]) : row;
+    int64_t dst = row;
+    if (kScatter) {
+      if (a.blk_base) {
+        // sorted row = first row of (block, expert) + number of earlier pairs of the block with that
+        // expert; a row group is made of whole warps, so the ballots below see converged warps
+        const int pair = (int)row * a.k + j;
+        const int e = a.topk_idx[pair];
+        const int blk = (int)(row / kRouteBlockTokens);
+        const int p0 = blk * kRouteBlockTokens * a.k;
+        int rank = 0;
+        for (int off = 0; off < kRouteBlockTokens * a.k; off += 32) {
+          const int pp = p0 + off + lane;
+          const bool m = pp < pair && a.topk_idx[pp] == e;
+          rank += __popc(__ballot_sync(0xffffffffu, m));
+        }
+        dst = a.blk_base[blk * a.E + e] + rank;
+        if (tg == 0) {
+          a.perm_out[pair] = (int32_t)dst;
+          a.inv_out[dst] = pair;
+        }
+      } else {
+        dst = a.perm[row * a.k + j];
+      }
+    }
     uint4* out = reinterpret_cast<uint4*>(a.q + dst * int64_t(a.d));
 #pragma unroll
     for (int u = 0; u < kUnits; ++u) {

@@ -156,9 +156,12 @@ __global__ void __launch_bounds__(kRmWarps * 32) route_topk_mma_kernel(const uin
                                                                      const float* __restrict__ bias, int E, int k,
                                                                      int norm_topk, int32_t* __restrict__ idx_out,
                                                                      float* __restrict__ w_out,
-                                                                     float* __restrict__ logits_out) {
+                                                                     float* __restrict__ logits_out,
+                                                                     int32_t* __restrict__ blk_hist) {
   __shared__ float s_part[kRmWarps][NE * 4][32];
   __shared__ float s_logits[16][NE * 8];
+  __shared__ int s_hist[NE * 8];                      // pairs per expert among this CTA's 16 tokens
+  if (threadIdx.x < NE * 8) s_hist[threadIdx.x] = 0;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
   const int64_t t0 = int64_t(blockIdx.x) * 16;
   const uint16_t* xa = x + min(t0 + g, T - 1) * int64_t(d) + t * 8;       // rows past the end alias the last row
@@ -277,23 +280,28 @@ __global__ void __launch_bounds__(kRmWarps * 32) route_topk_mma_kernel(const uin
         if (j < k) {
           idx_out[tok * k + j] = sel_i[j];
           w_out[tok * k + j] = ex[j] / denom;
+          atomicAdd(&s_hist[sel_i[j]], 1);
         }
     }
+  }
+  if (blk_hist) {                                      // input of the block-wise dispatch (dispatch.cu)
+    __syncthreads();
+    if (threadIdx.x < E) blk_hist[int64_t(blockIdx.x) * E + threadIdx.x] = s_hist[threadIdx.x];
   }
 }
 
 mote_status_t launch_route_topk(const void* x, int64_t T, int d, const float* Wr, const float* bias, int E,
-                                int k, int norm_topk, int32_t* idx, float* w, float* logits,
+                                int k, int norm_topk, int32_t* idx, float* w, float* logits, int32_t* blk_hist,
                                 cudaStream_t stream) {
   if (T == 0) return MOTE_OK;
   const uint16_t* xp = static_cast<const uint16_t*>(x);
   if (d % 32 == 0) {
     const unsigned blocks = (unsigned)((T + 15) / 16);
     const int ne = (E + 7) / 8;
-    if (ne <= 1) route_topk_mma_kernel<1><<<blocks, kRmWarps * 32, 0, stream>>>(xp, T, d, Wr, bias, E, k, norm_topk, idx, w, logits);
-    else if (ne <= 2) route_topk_mma_kernel<2><<<blocks, kRmWarps * 32, 0, stream>>>(xp, T, d, Wr, bias, E, k, norm_topk, idx, w, logits);
-    else if (ne <= 4) route_topk_mma_kernel<4><<<blocks, kRmWarps * 32, 0, stream>>>(xp, T, d, Wr, bias, E, k, norm_topk, idx, w, logits);
-    else route_topk_mma_kernel<8><<<blocks, kRmWarps * 32, 0, stream>>>(xp, T, d, Wr, bias, E, k, norm_topk, idx, w, logits);
+    if (ne <= 1) route_topk_mma_kernel<1><<<blocks, kRmWarps * 32, 0, stream>>>(xp, T, d, Wr, bias, E, k, norm_topk, idx, w, logits, blk_hist);
+    else if (ne <= 2) route_topk_mma_kernel<2><<<blocks, kRmWarps * 32, 0, stream>>>(xp, T, d, Wr, bias, E, k, norm_topk, idx, w, logits, blk_hist);
+    else if (ne <= 4) route_topk_mma_kernel<4><<<blocks, kRmWarps * 32, 0, stream>>>(xp, T, d, Wr, bias, E, k, norm_topk, idx, w, logits, blk_hist);
+    else route_topk_mma_kernel<8><<<blocks, kRmWarps * 32, 0, stream>>>(xp, T, d, Wr, bias, E, k, norm_topk, idx, w, logits, blk_hist);
   } else {
     const int per_cta = kRouteWarps * kRouteTok;
     const unsigned blocks = (unsigned)((T + per_cta - 1) / per_cta);
@@ -315,6 +323,6 @@ extern "C" mote_status_t mote_route_topk(const void* x_bf16, int64_t T, int64_t 
   if (T == 0) return MOTE_OK;
   if (!x_bf16 || !Wr || !topk_idx || !topk_w) return MOTE_ERR_NULL;
   if (!aligned16(x_bf16) || !aligned16(Wr)) return MOTE_ERR_ALIGN;
-  return launch_route_topk(x_bf16, T, (int)d, Wr, bias, E, k, norm_topk, topk_idx, topk_w, logits,
+  return launch_route_topk(x_bf16, T, (int)d, Wr, bias, E, k, norm_topk, topk_idx, topk_w, logits, nullptr,
                            static_cast<cudaStream_t>(stream));
 }
