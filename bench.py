@@ -99,7 +99,8 @@ class ClockSampler:
 
 # ncu dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the captures
 # summarised under profiles/ (null once the kernel has changed since, or where no capture exists)
-NCU_TRAFFIC_BYTES = {("c3-1", "gateup_ternary"): 70.70e6}
+NCU_TRAFFIC_BYTES = {("c2", "gateup_ternary"): 43.31e6, ("c4", "gateup_ternary"): 584.32e6,
+                     ("c3-1", "gateup_ternary"): 70.70e6}
 
 
 def stage_work(wl: synth.Workload, stage: str, stream_path: bool, experts_touched: float):
@@ -323,7 +324,7 @@ def run_ours(args):
         if is_stack:                                    # the oracle needs host-drawn weights: layer 0, scaled by the depth
             master = synth.master_layer(wl)
             x_bits = synth.tokens(wl)
-        cb = cpu_baseline(wl, master, x_bits, budget_s=20.0)
+        cb = cpu_baseline(wl, master, x_bits, budget_s=12.0)
         if is_stack:
             cb["value"] /= len(layers)
             cb["sample"] += f"; one layer timed, value divided by the {len(layers)} layers of the stack"
@@ -335,10 +336,15 @@ def run_ours(args):
 
 
 def cpu_baseline(wl, master, x_bits, budget_s: float, n_tokens: int | None = None):
-    """The oracle as it stands, on the host cores, on a bounded sample of the same workload."""
+    """The oracle as it stands, on the host cores, on a bounded sample of the same workload: a
+    short probe fixes the sample size so that the timed run takes about `budget_s` seconds."""
     from oracle import mote_oracle as O
     layer_or = O.build_layer(master)                     # offline step, not timed (as on the GPU)
-    n = n_tokens or min(wl.T, 256 if wl.d * wl.f < 8e6 else 64)
+    n0 = min(wl.T, 32)
+    t0 = time.perf_counter()
+    O.moe_forward(layer_or, x_bits, token_subset=np.arange(n0))
+    rate = n0 / max(time.perf_counter() - t0, 1e-6)
+    n = n_tokens or int(min(wl.T, max(n0, rate * budget_s)))
     sub = np.arange(n)
     t0 = time.perf_counter()
     O.moe_forward(layer_or, x_bits, token_subset=sub)
