@@ -44,8 +44,13 @@ typedef enum {
 enum { MOTE_DTYPE_F32 = 0, MOTE_DTYPE_BF16 = 1 };
 enum { MOTE_MAX_EXPERTS = 64, MOTE_MAX_TOPK = 8 };
 
-/* Which implementation the expert GEMMs use.  AUTO picks per shape; the others force one path
- * (used by the tests to check every path against the oracle). */
+/* Which implementation runs the layer.  AUTO picks per shape; the others force one path (used by
+ * the tests to check every path against the oracle).
+ *   STREAM  decode, T <= 64 with d % 64 == 0, f % 64 == 0, d <= 16384, T*k <= 512: the weights are
+ *           streamed once from HBM through registers into warp-level MMAs
+ *   TENSOR  d % 128 == 0 and f % 128 == 0: tcgen05 GEMMs (int8 x 2-bit routed, bf16 shared)
+ *   SIMT    any d, f that are multiples of 16: CUDA-core GEMMs
+ * AUTO takes the first of these whose conditions hold. */
 enum { MOTE_PATH_AUTO = 0, MOTE_PATH_SIMT = 1, MOTE_PATH_TENSOR = 2, MOTE_PATH_STREAM = 3 };
 
 const char* mote_status_string(mote_status_t st);
@@ -187,7 +192,7 @@ size_t mote_workspace_bytes(int d, int f, int E, int k, int64_t T_max);
  * h = bf16_rn(u * silu(g)) with silu evaluated by a fixed fp32 sequence, so that the integer
  * stages that follow are reproducible bit for bit.
  * T = 0 is a no-op.  Errors: d%16, f%16 != 0, E/k out of range -> ERR_SHAPE; ERR_WORKSPACE;
- * ERR_ALIGN; path = MOTE_PATH_TENSOR with d%128 or f%128 != 0 -> ERR_SHAPE.
+ * ERR_ALIGN; a forced path whose conditions (see MOTE_PATH_*) do not hold -> ERR_SHAPE.
  */
 mote_status_t mote_moe_forward(const mote_layer_t* L, const void* x_bf16,
                                const void* residual_bf16, int64_t T, void* out_bf16,
@@ -237,7 +242,10 @@ mote_status_t mote_stack_forward(const mote_layer_t* layers_host, int n_layers, 
  * and writes the device time of each stage, in milliseconds, to stage_ms_host[MOTE_N_STAGES]:
  *   0 route (Eq. 3)   1 dispatch   2 Q_a(x) (Eq. 8)   3 gate/up ternary GEMM (Eq. 6)   4 Q_a(h)
  *   5 down ternary GEMM (Eq. 5)   6 shared gate/up   7 shared down (Eq. 2)   8 combine (Eq. 2, 4)
- * A stage that a fused path folds into its neighbour reports 0.  Stages run back to back on one
+ * A stage that a path folds into its neighbour reports 0: the tensor path does the combine in the
+ * shared-down epilogue (stage 7); the decode path reports its prologue (Q_a(x), router, dispatch)
+ * as stage 0 and its two streaming kernels, which cover the routed AND the shared expert, as
+ * stages 3 and 5.  Stages run back to back on one
  * stream here even if mote_moe_forward overlaps some of them. */
 enum { MOTE_N_STAGES = 9 };
 mote_status_t mote_moe_forward_profile(const mote_layer_t* L, const void* x_bf16,
