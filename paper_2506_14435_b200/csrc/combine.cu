@@ -13,6 +13,7 @@ __global__ void __launch_bounds__(256) combine_kernel(const float* __restrict__ 
                                                       uint16_t* out) {
   const int vec_per_row = d / 8;
   const int64_t total = T * vec_per_row;
+  pdl_wait();                            // no-op unless launched as a programmatic dependent
   const int64_t stride = int64_t(gridDim.x) * blockDim.x;
   for (int64_t i = int64_t(blockIdx.x) * blockDim.x + threadIdx.x; i < total; i += stride) {
     const int64_t t = i / vec_per_row;
@@ -48,12 +49,17 @@ __global__ void __launch_bounds__(256) combine_kernel(const float* __restrict__ 
 }
 
 mote_status_t launch_combine(const float* s, const float* y, const float* w, const int32_t* perm,
-                             const void* residual, int64_t T, int d, int k, void* out_bf16, cudaStream_t stream) {
+                             const void* residual, int64_t T, int d, int k, void* out_bf16, cudaStream_t stream,
+                             bool pdl) {
   if (T == 0) return MOTE_OK;
   const int64_t total = T * (d / 8);
   const unsigned blocks = (unsigned)std::min<int64_t>((total + 255) / 256, 148 * 16);
-  combine_kernel<<<blocks, 256, 0, stream>>>(s, y, w, perm, static_cast<const uint16_t*>(residual), T, d, k,
-                                             static_cast<uint16_t*>(out_bf16));
+  if (pdl)
+    MOTE_CUDA_OK(launch_pdl(combine_kernel, dim3(blocks), dim3(256), 0, stream, s, y, w, perm,
+                            static_cast<const uint16_t*>(residual), T, d, k, static_cast<uint16_t*>(out_bf16)));
+  else
+    combine_kernel<<<blocks, 256, 0, stream>>>(s, y, w, perm, static_cast<const uint16_t*>(residual), T, d, k,
+                                               static_cast<uint16_t*>(out_bf16));
   ++g_launch_count;
   MOTE_LAUNCH_OK();
   return MOTE_OK;

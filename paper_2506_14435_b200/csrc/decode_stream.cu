@@ -88,6 +88,7 @@ __global__ void __launch_bounds__(256) decode_prologue_kernel(DecodePrologueArgs
   const int t = blockIdx.x;
   const int d = a.d, n_vec = d / 8, n_units = d / 16;
   const uint4* src = reinterpret_cast<const uint4*>(a.x + int64_t(t) * d);
+  pdl_trigger();                         // the gate/up kernel may start on the shared expert right away
 
   float amax = 0.0f;
   for (int v = tid; v < n_vec; v += 256) {
@@ -521,13 +522,22 @@ __global__ void __launch_bounds__(kGuWarps * 32) decode_gateup_kernel(DecodeGate
   __shared__ ExpertList s_list;
   __shared__ float s_part[kGuWarps * NTB * 4 * 32];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  if (warp == 0) build_expert_list(a.c.offsets, a.c.E, &s_list);
-  __syncthreads();
   const int tiles = a.c.f / 8;
   const int quads = (tiles + kGuWarps - 1) / kGuWarps;
   const int n_shared = tiles;
-  const int n_items = n_shared + s_list.n * quads;
-  for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+  // The shared expert needs nothing from the prologue kernel, so its items run before the wait on
+  // that kernel; the routing tables are read only when the CTA reaches its first routed item.
+  bool routed_ready = false;
+  int n_items = n_shared;
+  for (int item = blockIdx.x;; item += gridDim.x) {
+    if (item >= n_shared && !routed_ready) {
+      pdl_wait();
+      if (warp == 0) build_expert_list(a.c.offsets, a.c.E, &s_list);
+      __syncthreads();
+      n_items = n_shared + s_list.n * quads;
+      routed_ready = true;
+    }
+    if (item >= n_items) break;
     if (item < n_shared) {
       gateup_shared_tile<NTB>(a, item, warp, lane, s_part);
     } else {
@@ -664,6 +674,7 @@ __global__ void __launch_bounds__(kDownWarps * 32) decode_down_kernel(DecodeDown
   __shared__ ExpertList s_list;
   extern __shared__ float s_part[];                       // kDownWarps * NTB * 4 * 32 floats
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  pdl_wait();                            // Q_a(h) has completed
   if (warp == 0) build_expert_list(a.c.offsets, a.c.E, &s_list);
   __syncthreads();
   const int tiles = a.c.d / 16;
@@ -738,10 +749,10 @@ mote_status_t launch_decode_stream(const DecodeStreamArgs& p, int phase, cudaStr
     const int tiles = f / 8, quads = (tiles + kGuWarps - 1) / kGuWarps;
     const int max_items = tiles + std::min<int>(E, T * k) * quads;
     const int grid = std::min(max_items, sms * 12);
-    if (ntb == 1) decode_gateup_kernel<1><<<grid, kGuWarps * 32, 0, stream>>>(ga);
-    else if (ntb == 2) decode_gateup_kernel<2><<<grid, kGuWarps * 32, 0, stream>>>(ga);
-    else if (ntb == 4) decode_gateup_kernel<4><<<grid, kGuWarps * 32, 0, stream>>>(ga);
-    else decode_gateup_kernel<8><<<grid, kGuWarps * 32, 0, stream>>>(ga);
+    if (ntb == 1) MOTE_CUDA_OK(launch_pdl(decode_gateup_kernel<1>, dim3(grid), dim3(kGuWarps * 32), 0, stream, ga));
+    else if (ntb == 2) MOTE_CUDA_OK(launch_pdl(decode_gateup_kernel<2>, dim3(grid), dim3(kGuWarps * 32), 0, stream, ga));
+    else if (ntb == 4) MOTE_CUDA_OK(launch_pdl(decode_gateup_kernel<4>, dim3(grid), dim3(kGuWarps * 32), 0, stream, ga));
+    else MOTE_CUDA_OK(launch_pdl(decode_gateup_kernel<8>, dim3(grid), dim3(kGuWarps * 32), 0, stream, ga));
     ++g_launch_count;
     MOTE_LAUNCH_OK();
     return MOTE_OK;
@@ -760,10 +771,10 @@ mote_status_t launch_decode_stream(const DecodeStreamArgs& p, int phase, cudaStr
     MOTE_CUDA_OK(cudaFuncSetAttribute(decode_down_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 65536));
     down_attr_set = true;
   }
-  if (ntb == 1) decode_down_kernel<1><<<grid, kDownWarps * 32, smem, stream>>>(da);
-  else if (ntb == 2) decode_down_kernel<2><<<grid, kDownWarps * 32, smem, stream>>>(da);
-  else if (ntb == 4) decode_down_kernel<4><<<grid, kDownWarps * 32, smem, stream>>>(da);
-  else decode_down_kernel<8><<<grid, kDownWarps * 32, smem, stream>>>(da);
+  if (ntb == 1) MOTE_CUDA_OK(launch_pdl(decode_down_kernel<1>, dim3(grid), dim3(kDownWarps * 32), smem, stream, da));
+  else if (ntb == 2) MOTE_CUDA_OK(launch_pdl(decode_down_kernel<2>, dim3(grid), dim3(kDownWarps * 32), smem, stream, da));
+  else if (ntb == 4) MOTE_CUDA_OK(launch_pdl(decode_down_kernel<4>, dim3(grid), dim3(kDownWarps * 32), smem, stream, da));
+  else MOTE_CUDA_OK(launch_pdl(decode_down_kernel<8>, dim3(grid), dim3(kDownWarps * 32), smem, stream, da));
   ++g_launch_count;
   MOTE_LAUNCH_OK();
   return MOTE_OK;

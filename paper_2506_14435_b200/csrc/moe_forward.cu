@@ -216,13 +216,13 @@ extern "C" mote_status_t mote_moe_forward(const mote_layer_t* L, const void* x, 
     st = launch_decode_stream(ds, 1, stream);                 // routed and shared gate/up
     if (st) return st;
     stage_mark(4, stream);
-    st = launch_quant_rows_known_beta(h, P, f, qh, beta_h, rowsum_h, 1, stream);
+    st = launch_quant_rows_known_beta(h, P, f, qh, beta_h, rowsum_h, 1, stream, true);
     if (st) return st;
     stage_mark(5, stream);
     st = launch_decode_stream(ds, 2, stream);                 // routed and shared down
     if (st) return st;
     stage_mark(6, stream); stage_mark(7, stream); stage_mark(8, stream);
-    st = launch_combine(s, y, topk_w, perm, residual, T, d, k, out, stream);
+    st = launch_combine(s, y, topk_w, perm, residual, T, d, k, out, stream, true);
     if (st) return st;
     stage_mark(9, stream);
     if (taps) {

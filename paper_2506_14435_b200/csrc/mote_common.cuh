@@ -19,6 +19,33 @@
 
 namespace mote {
 
+// ---------------------------------------------------------------------------------------------
+// Programmatic dependent launch: a kernel launched with launch_pdl may start while the kernel
+// before it on the stream is still running; it calls pdl_wait() before it touches anything that
+// kernel writes (the wait returns once the earlier kernel has completed and its writes are
+// visible; in a kernel launched the ordinary way it returns at once).  A kernel calls
+// pdl_trigger() to let its successor start early; without it the successor starts as the kernel's
+// CTAs exit, which still hides the successor's launch latency.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+static inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                     Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 constexpr float kEpsScale = 1e-5f;  // lower clamp of alpha (Eq. 9) and beta (Eq. 8)
 
 static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }

@@ -76,8 +76,9 @@ mote_status_t launch_ternary_umma(const TernaryGemmArgs& a, bool gateup, const i
 
 // Q_a(h) for rows whose absmax is already known: beta_bits holds max |h| per row (raw bits);
 // writes q (k-interleaved if asked), the clamped beta in place, and accumulates rowsum (zeroed).
+// pdl: launch as a programmatic dependent of the kernel before it on the stream (decode path)
 mote_status_t launch_quant_rows_known_beta(const void* h_bf16, int64_t rows, int n, int8_t* q, float* beta,
-                                           int32_t* rowsum, int interleave, cudaStream_t stream);
+                                           int32_t* rowsum, int interleave, cudaStream_t stream, bool pdl = false);
 // comb (down projection only, may be null): fold the combine of Eq. 2 / Eq. 4 into the epilogue and
 // write the layer output directly; `out` (fp32 s) may then be null.
 struct CombineArgs {
@@ -118,6 +119,6 @@ mote_status_t launch_rms_norm(const void* x, int64_t T, int d, float eps, void* 
 // out = [residual +] s + sum_j w_j * y[perm[t*k+j]]
 mote_status_t launch_combine(const float* s, const float* y, const float* w, const int32_t* perm,
                              const void* residual, int64_t T, int d, int k, void* out_bf16,
-                             cudaStream_t stream);
+                             cudaStream_t stream, bool pdl = false);
 
 }  // namespace mote

@@ -148,6 +148,7 @@ __global__ void __launch_bounds__(256) quant_rows_known_beta_kernel(const uint4*
   const int lane = threadIdx.x & 31;
   const int64_t stride = int64_t(gridDim.x) * blockDim.x;
   const int64_t first = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
+  pdl_wait();                            // no-op unless launched as a programmatic dependent
   for (int64_t base = first - lane; base < n_units_total; base += stride) {
     const int64_t u = base + lane;
     const bool ok = u < n_units_total;
@@ -182,13 +183,18 @@ __global__ void __launch_bounds__(256) quant_rows_known_beta_kernel(const uint4*
 }
 
 mote_status_t launch_quant_rows_known_beta(const void* h_bf16, int64_t rows, int n, int8_t* q, float* beta,
-                                           int32_t* rowsum, int interleave, cudaStream_t stream) {
+                                           int32_t* rowsum, int interleave, cudaStream_t stream, bool pdl) {
   if (rows == 0) return MOTE_OK;
   const int units_per_row = n / 16;
   const int64_t total = rows * units_per_row;
   const unsigned blocks = (unsigned)std::min<int64_t>((total + 255) / 256, 148 * 8);
-  quant_rows_known_beta_kernel<<<blocks, 256, 0, stream>>>(static_cast<const uint4*>(h_bf16), total, units_per_row,
-                                                           reinterpret_cast<uint4*>(q), beta, rowsum, interleave);
+  if (pdl)
+    MOTE_CUDA_OK(launch_pdl(quant_rows_known_beta_kernel, dim3(blocks), dim3(256), 0, stream,
+                            static_cast<const uint4*>(h_bf16), total, units_per_row, reinterpret_cast<uint4*>(q), beta,
+                            rowsum, interleave));
+  else
+    quant_rows_known_beta_kernel<<<blocks, 256, 0, stream>>>(static_cast<const uint4*>(h_bf16), total, units_per_row,
+                                                             reinterpret_cast<uint4*>(q), beta, rowsum, interleave);
   ++g_launch_count;
   MOTE_LAUNCH_OK();
   return MOTE_OK;
