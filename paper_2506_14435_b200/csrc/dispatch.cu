@@ -131,6 +131,7 @@ __global__ void __launch_bounds__(kDispatchThreads) dispatch_scan_kernel(const i
   __shared__ int s_first[MOTE_MAX_EXPERTS];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   constexpr int kPer = 16;                             // blocks per lane and chunk: 16 independent loads
+  pdl_wait();                                          // the router's block counts are complete
   // totals per expert (two rounds of 32 warps cover MOTE_MAX_EXPERTS = 64)
 #pragma unroll
   for (int r = 0; r < 2; ++r) {
@@ -212,8 +213,8 @@ __global__ void __launch_bounds__(kDispatchThreads) dispatch_scan_kernel(const i
 
 mote_status_t launch_dispatch_scan(const int32_t* blk_hist, int n_blk, int E, int32_t* offsets, int32_t* blk_base,
                                    int4* tiles_routed, int4* tiles_shared, int64_t T, cudaStream_t stream) {
-  dispatch_scan_kernel<<<1, kDispatchThreads, 0, stream>>>(blk_hist, n_blk, E, offsets, blk_base, tiles_routed,
-                                                           tiles_shared, (int)T);
+  MOTE_CUDA_OK(launch_pdl(dispatch_scan_kernel, dim3(1), dim3(kDispatchThreads), 0, stream, blk_hist, n_blk, E, offsets,
+                          blk_base, tiles_routed, tiles_shared, (int)T));
   ++g_launch_count;
   MOTE_LAUNCH_OK();
   return MOTE_OK;

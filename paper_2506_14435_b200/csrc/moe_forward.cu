@@ -272,7 +272,9 @@ extern "C" mote_status_t mote_moe_forward(const mote_layer_t* L, const void* x, 
   qa.perm = perm; qa.k = k; qa.interleave = interleave;
   if (blockwise) {
     qa.topk_idx = topk_idx; qa.blk_base = blk_base; qa.E = E; qa.perm_out = perm; qa.inv_out = inv;
+    qa.zero_u32 = reinterpret_cast<uint32_t*>(beta_h); qa.zero_i32 = rowsum_h;
   }
+  const bool pdl = blockwise;    // from here on every kernel is a programmatic dependent of the one before
   st = launch_quant_act(qa, true, stream);
   if (st) return st;
   stage_mark(3, stream);
@@ -281,10 +283,10 @@ extern "C" mote_status_t mote_moe_forward(const mote_layer_t* L, const void* x, 
   g1.qa = qx; g1.beta = beta_x; g1.offsets = offsets; g1.w0 = L->gate_packed; g1.w1 = L->up_packed;
   g1.alpha0 = L->alpha_gate; g1.alpha1 = L->alpha_up; g1.E = E; g1.N = f; g1.K = d; g1.P = P;
   g1.h_bf16 = h; g1.acc0_tap = taps ? taps->acc_gate : nullptr; g1.acc1_tap = taps ? taps->acc_up : nullptr;
-  if (tensor)   // beta_h (atomicMax target) and rowsum_h (atomicAdd target) are adjacent
+  if (tensor && !blockwise)   // beta_h (atomicMax target) and rowsum_h (atomicAdd target) are adjacent
     MOTE_CUDA_OK(cudaMemsetAsync(beta_h, 0, (pl.rowsum_h - pl.beta_h) + size_t(P) * 4, stream));
   st = tensor ? launch_ternary_umma(g1, true, tiles_routed, max_mtiles_routed, rowsum_x,
-                                    reinterpret_cast<uint32_t*>(beta_h), status, stream)
+                                    reinterpret_cast<uint32_t*>(beta_h), status, stream, pdl)
               : launch_ternary_gateup_simt(g1, stream);
   if (st) return st;
   stage_mark(4, stream);
@@ -292,7 +294,7 @@ extern "C" mote_status_t mote_moe_forward(const mote_layer_t* L, const void* x, 
   QuantActArgs qb{};
   qb.x = h; qb.T = P; qb.d = f; qb.ldx = f; qb.q = qh; qb.beta = beta_h; qb.rowsum = rowsum_h;
   qb.perm = nullptr; qb.k = 1; qb.interleave = interleave;
-  st = tensor ? launch_quant_rows_known_beta(h, P, f, qh, beta_h, rowsum_h, interleave, stream)
+  st = tensor ? launch_quant_rows_known_beta(h, P, f, qh, beta_h, rowsum_h, interleave, stream, pdl)
               : launch_quant_act(qb, false, stream);
   if (st) return st;
   stage_mark(5, stream);
@@ -300,13 +302,13 @@ extern "C" mote_status_t mote_moe_forward(const mote_layer_t* L, const void* x, 
   TernaryGemmArgs g2{};
   g2.qa = qh; g2.beta = beta_h; g2.offsets = offsets; g2.w0 = L->down_packed; g2.alpha0 = L->alpha_down;
   g2.E = E; g2.N = d; g2.K = f; g2.P = P; g2.y = y; g2.acc0_tap = taps ? taps->acc_down : nullptr;
-  st = tensor ? launch_ternary_umma(g2, false, tiles_routed, max_mtiles_routed, rowsum_h, nullptr, status, stream)
+  st = tensor ? launch_ternary_umma(g2, false, tiles_routed, max_mtiles_routed, rowsum_h, nullptr, status, stream, pdl)
               : launch_ternary_down_simt(g2, stream);
   if (st) return st;
   stage_mark(6, stream);
   // S7 shared expert
   st = tensor ? launch_shared_umma(x, L->sh_gate, L->sh_up, true, T, d, f, hs, tiles_shared, max_mtiles_shared,
-                                   status, nullptr, stream)
+                                   status, nullptr, stream, pdl)
               : launch_shared_gateup_simt(x, L->sh_gate, L->sh_up, T, d, f, hs, stream);
   if (st) return st;
   stage_mark(7, stream);
@@ -315,7 +317,7 @@ extern "C" mote_status_t mote_moe_forward(const mote_layer_t* L, const void* x, 
     // shared output is written only when a tap asks for it
     CombineArgs cb{y, topk_w, perm, residual, out, k};
     st = launch_shared_umma(hs, L->sh_down, nullptr, false, T, f, d, (taps && taps->shared_out) ? s : nullptr,
-                            tiles_shared, max_mtiles_shared, status, &cb, stream);
+                            tiles_shared, max_mtiles_shared, status, &cb, stream, pdl);
     if (st) return st;
     stage_mark(8, stream);
   } else {

@@ -21,6 +21,7 @@ struct QuantActArgs {
   // top-k indices and the per-block bases, and written to perm_out / inv_out
   const int32_t* topk_idx; const int32_t* blk_base; int E;
   int32_t* perm_out; int32_t* inv_out;
+  uint32_t* zero_u32; int32_t* zero_i32;   // optional [rows] arrays cleared at every destination row
   int k;
   int interleave;       // 1: store each unit of 16 codes k-interleaved
   int group;            // threads per row (set by the launcher)
@@ -72,7 +73,7 @@ mote_status_t launch_ternary_down_simt(const TernaryGemmArgs& a, cudaStream_t st
 // beta_out_bits (gate/up only, may be null): per row, atomicMax of the bits of |h| (must be zeroed).
 mote_status_t launch_ternary_umma(const TernaryGemmArgs& a, bool gateup, const int4* tiles, int max_mtiles,
                                   const int32_t* rowsum, uint32_t* beta_out_bits, uint32_t* status,
-                                  cudaStream_t stream);
+                                  cudaStream_t stream, bool pdl = false);
 
 // Q_a(h) for rows whose absmax is already known: beta_bits holds max |h| per row (raw bits);
 // writes q (k-interleaved if asked), the clamped beta in place, and accumulates rowsum (zeroed).
@@ -86,7 +87,7 @@ struct CombineArgs {
 };
 mote_status_t launch_shared_umma(const void* act, const void* w0, const void* w1, bool gateup, int64_t T, int K,
                                  int N, void* out, const int4* tiles, int max_mtiles, uint32_t* status,
-                                 const CombineArgs* comb, cudaStream_t stream);
+                                 const CombineArgs* comb, cudaStream_t stream, bool pdl = false);
 
 // CUDA-core bf16 GEMMs of the shared expert.
 mote_status_t launch_shared_gateup_simt(const void* x, const void* Wg, const void* Wu, int64_t T, int d,

@@ -100,6 +100,8 @@ __global__ void __launch_bounds__(256) quant_act_kernel(QuantActArgs a) {
   }
   if (!row_ok) return;
 
+  // everything above depends on x only; the routing of the kernels before this one is needed from here on
+  if (kScatter) pdl_wait();
   const int n_dst = kScatter ? a.k : 1;
   for (int j = 0; j < n_dst; ++j) {
     int64_t dst = row;
@@ -121,6 +123,10 @@ __global__ void __launch_bounds__(256) quant_act_kernel(QuantActArgs a) {
         if (tg == 0) {
           a.perm_out[pair] = (int32_t)dst;
           a.inv_out[dst] = pair;
+          if (a.zero_u32) {                              // targets of the gate/up epilogue's atomics
+            a.zero_u32[dst] = 0u;
+            a.zero_i32[dst] = 0;
+          }
         }
       } else {
         dst = a.perm[row * a.k + j];
@@ -214,7 +220,9 @@ mote_status_t launch_quant_act(const QuantActArgs& a, bool scatter, cudaStream_t
   const unsigned blocks = (unsigned)((a.T + rows_per_cta - 1) / rows_per_cta);
 #define MOTE_QA_LAUNCH(U)                                                          \
   do {                                                                             \
-    if (scatter) quant_act_kernel<U, true><<<blocks, threads, 0, stream>>>(args);  \
+    if (scatter && args.blk_base)                                                   \
+      MOTE_CUDA_OK(launch_pdl(quant_act_kernel<U, true>, dim3(blocks), dim3(threads), 0, stream, args)); \
+    else if (scatter) quant_act_kernel<U, true><<<blocks, threads, 0, stream>>>(args);  \
     else quant_act_kernel<U, false><<<blocks, threads, 0, stream>>>(args);         \
   } while (0)
   if (upt <= 1) MOTE_QA_LAUNCH(1);

@@ -128,8 +128,6 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
   volatile int* abort_flag = &bars->abort_flag;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int n_mtiles = a.tiles[0].x;
-  const int n_items = n_mtiles * a.n_ntiles;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < 4; ++s) {
@@ -157,6 +155,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = bars->tmem_base;
+  pdl_wait();                              // set-up above overlaps the tail of the kernel before this one
+  const int n_mtiles = a.tiles[0].x;
+  const int n_items = n_mtiles * a.n_ntiles;
 
   if (warp == 0) {
     // ---------------------------------------------------------------- token-operand producer
@@ -534,7 +535,7 @@ static int pick_bn(int N) {
 
 template <int MODE>
 static mote_status_t launch_umma(const CUtensorMap& ta, const CUtensorMap& tb0, const CUtensorMap& tb1,
-                                 const UmmaArgs& a, int max_items, cudaStream_t stream) {
+                                 const UmmaArgs& a, int max_items, cudaStream_t stream, bool pdl) {
   using TR = ModeTraits<MODE>;
   static bool attr_set = false;
   if (!attr_set) {
@@ -545,7 +546,8 @@ static mote_status_t launch_umma(const CUtensorMap& ta, const CUtensorMap& tb0, 
   MOTE_CUDA_OK(cudaGetDevice(&dev));
   MOTE_CUDA_OK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
   const int grid = std::max(1, std::min(sms, max_items));
-  umma_gemm_kernel<MODE><<<grid, kThreads, TR::kSmem, stream>>>(ta, tb0, tb1, a);
+  if (pdl) MOTE_CUDA_OK(launch_pdl(umma_gemm_kernel<MODE>, dim3(grid), dim3(kThreads), TR::kSmem, stream, ta, tb0, tb1, a));
+  else umma_gemm_kernel<MODE><<<grid, kThreads, TR::kSmem, stream>>>(ta, tb0, tb1, a);
   ++g_launch_count;
   MOTE_LAUNCH_OK();
   return MOTE_OK;
@@ -553,7 +555,7 @@ static mote_status_t launch_umma(const CUtensorMap& ta, const CUtensorMap& tb0, 
 
 mote_status_t launch_ternary_umma(const TernaryGemmArgs& g, bool gateup, const int4* tiles, int max_mtiles,
                                   const int32_t* rowsum, uint32_t* beta_out_bits, uint32_t* status,
-                                  cudaStream_t stream) {
+                                  cudaStream_t stream, bool pdl) {
   if (g.P == 0) return MOTE_OK;
   CUtensorMap ta, tb0, tb1;
   const int bn = gateup ? 256 : pick_bn(g.N);
@@ -580,13 +582,13 @@ mote_status_t launch_ternary_umma(const TernaryGemmArgs& g, bool gateup, const i
   a.beta_out_bits = gateup ? beta_out_bits : nullptr;
   a.status = status;
   const int max_items = max_mtiles * a.n_ntiles;
-  return gateup ? launch_umma<MODE_T_GATEUP>(ta, tb0, tb1, a, max_items, stream)
-                : launch_umma<MODE_T_DOWN>(ta, tb0, tb1, a, max_items, stream);
+  return gateup ? launch_umma<MODE_T_GATEUP>(ta, tb0, tb1, a, max_items, stream, pdl)
+                : launch_umma<MODE_T_DOWN>(ta, tb0, tb1, a, max_items, stream, pdl);
 }
 
 mote_status_t launch_shared_umma(const void* act, const void* w0, const void* w1, bool gateup, int64_t T, int K,
                                  int N, void* out, const int4* tiles, int max_mtiles, uint32_t* status,
-                                 const CombineArgs* comb, cudaStream_t stream) {
+                                 const CombineArgs* comb, cudaStream_t stream, bool pdl) {
   if (T == 0) return MOTE_OK;
   CUtensorMap ta, tb0, tb1;
   const int bn = gateup ? 256 : pick_bn(N);
@@ -614,8 +616,8 @@ mote_status_t launch_shared_umma(const void* act, const void* w0, const void* w1
     a.comb_k = comb->k;
   }
   const int max_items = max_mtiles * a.n_ntiles;
-  return gateup ? launch_umma<MODE_B_GATEUP>(ta, tb0, tb1, a, max_items, stream)
-                : launch_umma<MODE_B_DOWN>(ta, tb0, tb1, a, max_items, stream);
+  return gateup ? launch_umma<MODE_B_GATEUP>(ta, tb0, tb1, a, max_items, stream, pdl)
+                : launch_umma<MODE_B_DOWN>(ta, tb0, tb1, a, max_items, stream, pdl);
 }
 
 }  // namespace mote
