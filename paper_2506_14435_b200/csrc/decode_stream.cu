@@ -674,14 +674,21 @@ __global__ void __launch_bounds__(kDownWarps * 32) decode_down_kernel(DecodeDown
   __shared__ ExpertList s_list;
   extern __shared__ float s_part[];                       // kDownWarps * NTB * 4 * 32 floats
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  pdl_wait();                            // Q_a(h) has completed
+  // This kernel is let in as soon as Q_a(h) has STARTED (which is after the gate/up kernel and
+  // the prologue have completed): the dispatch tables and h_shared are there, and the shared
+  // expert's slices are streamed while Q_a(h) runs.  The routed items wait for it.
   if (warp == 0) build_expert_list(a.c.offsets, a.c.E, &s_list);
   __syncthreads();
   const int tiles = a.c.d / 16;
   const int n_shared = tiles;
   const int n_items = n_shared + s_list.n * tiles;
   int* ip = reinterpret_cast<int*>(s_part);
+  bool waited = false;
   for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+    if (item >= n_shared && !waited) {
+      pdl_wait();                          // Q_a(h) has completed
+      waited = true;
+    }
     if (item < n_shared) {
       down_shared_tile<NTB>(a, item, warp, lane, s_part);
     } else {
@@ -695,6 +702,7 @@ __global__ void __launch_bounds__(kDownWarps * 32) decode_down_kernel(DecodeDown
       else down_routed_tile<(NTB >= 8 ? 8 : 1)>(a, e, tile, warp, lane, ip);
     }
   }
+  if (!waited) pdl_wait();                 // no CTA leaves before the kernels ahead of it are complete
 }
 
 // ------------------------------------------------------------------------------------------------

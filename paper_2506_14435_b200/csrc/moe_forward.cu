@@ -216,7 +216,7 @@ extern "C" mote_status_t mote_moe_forward(const mote_layer_t* L, const void* x, 
     st = launch_decode_stream(ds, 1, stream);                 // routed and shared gate/up
     if (st) return st;
     stage_mark(4, stream);
-    st = launch_quant_rows_known_beta(h, P, f, qh, beta_h, rowsum_h, 1, stream, true);
+    st = launch_quant_rows_known_beta(h, P, f, qh, beta_h, rowsum_h, 1, stream, true, true);
     if (st) return st;
     stage_mark(5, stream);
     st = launch_decode_stream(ds, 2, stream);                 // routed and shared down

@@ -79,7 +79,8 @@ mote_status_t launch_ternary_umma(const TernaryGemmArgs& a, bool gateup, const i
 // writes q (k-interleaved if asked), the clamped beta in place, and accumulates rowsum (zeroed).
 // pdl: launch as a programmatic dependent of the kernel before it on the stream (decode path)
 mote_status_t launch_quant_rows_known_beta(const void* h_bf16, int64_t rows, int n, int8_t* q, float* beta,
-                                           int32_t* rowsum, int interleave, cudaStream_t stream, bool pdl = false);
+                                           int32_t* rowsum, int interleave, cudaStream_t stream, bool pdl = false,
+                                           bool early_trigger = false);
 // comb (down projection only, may be null): fold the combine of Eq. 2 / Eq. 4 into the epilogue and
 // write the layer output directly; `out` (fp32 s) may then be null.
 struct CombineArgs {

@@ -150,11 +150,14 @@ __global__ void __launch_bounds__(256) quant_act_kernel(QuantActArgs a) {
 __global__ void __launch_bounds__(256) quant_rows_known_beta_kernel(const uint4* __restrict__ h, int64_t n_units_total,
                                                                     int units_per_row, uint4* __restrict__ q,
                                                                     float* beta, int32_t* __restrict__ rowsum,
-                                                                    int interleave) {
+                                                                    int interleave, int early_trigger) {
   const int lane = threadIdx.x & 31;
   const int64_t stride = int64_t(gridDim.x) * blockDim.x;
   const int64_t first = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
   pdl_wait();                            // no-op unless launched as a programmatic dependent
+  // decode path: the down kernel may start on work that does not need this kernel's output.  (Not
+  // for the tensor path: its persistent GEMM CTAs would take this kernel's registers away.)
+  if (early_trigger) pdl_trigger();
   for (int64_t base = first - lane; base < n_units_total; base += stride) {
     const int64_t u = base + lane;
     const bool ok = u < n_units_total;
@@ -189,7 +192,8 @@ __global__ void __launch_bounds__(256) quant_rows_known_beta_kernel(const uint4*
 }
 
 mote_status_t launch_quant_rows_known_beta(const void* h_bf16, int64_t rows, int n, int8_t* q, float* beta,
-                                           int32_t* rowsum, int interleave, cudaStream_t stream, bool pdl) {
+                                           int32_t* rowsum, int interleave, cudaStream_t stream, bool pdl,
+                                           bool early_trigger) {
   if (rows == 0) return MOTE_OK;
   const int units_per_row = n / 16;
   const int64_t total = rows * units_per_row;
@@ -197,10 +201,10 @@ mote_status_t launch_quant_rows_known_beta(const void* h_bf16, int64_t rows, int
   if (pdl)
     MOTE_CUDA_OK(launch_pdl(quant_rows_known_beta_kernel, dim3(blocks), dim3(256), 0, stream,
                             static_cast<const uint4*>(h_bf16), total, units_per_row, reinterpret_cast<uint4*>(q), beta,
-                            rowsum, interleave));
+                            rowsum, interleave, early_trigger ? 1 : 0));
   else
     quant_rows_known_beta_kernel<<<blocks, 256, 0, stream>>>(static_cast<const uint4*>(h_bf16), total, units_per_row,
-                                                             reinterpret_cast<uint4*>(q), beta, rowsum, interleave);
+                                                             reinterpret_cast<uint4*>(q), beta, rowsum, interleave, 0);
   ++g_launch_count;
   MOTE_LAUNCH_OK();
   return MOTE_OK;
