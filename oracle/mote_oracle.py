@@ -290,6 +290,88 @@ def shared_ffn(x_bf16, Wg_bf16, Wu_bf16, Wd_bf16) -> np.ndarray:
 
 
 # --------------------------------------------------------------------------------------------
+# Section 4.3  post-training quantization of the shared expert: round-to-nearest (RTN), weight-only
+# --------------------------------------------------------------------------------------------
+
+
+def rtn_quantize(W: np.ndarray, bits: int):
+    """RTN absmax quantizer of a weight matrix W[m, n] to `bits`-bit signed integers (8 or 4), one
+    scale per output row (the absmax form of Eq. 8-10 applied to the rows of W):
+
+        qmax   = 2^(bits-1) - 1                        127 or 7
+        beta_r = max(max_j |W[r, j]|, 1e-5)
+        q[r,j] = RoundClip(qmax * W[r, j] / beta_r, -qmax, qmax)
+        scale_r = beta_r / qmax                        dequantized weight = scale_r * q[r, j]
+
+    Written as single fp32 operations (one multiply, one true division, round half to even) so
+    that the integer codes are reproducible bit for bit.  Returns (q int8 [m, n], scale f32 [m])."""
+    if bits not in (8, 4):
+        raise ValueError("bits must be 8 or 4")
+    W = np.asarray(W, dtype=np.float32)
+    qmax = F32(2 ** (bits - 1) - 1)
+    beta = np.maximum(np.max(np.abs(W), axis=1), EPS_SCALE).astype(np.float32)
+    t = qmax * W
+    q = round_clip(t / beta[:, None], -float(qmax), float(qmax)).astype(np.int8)
+    scale = (beta / qmax).astype(np.float32)
+    return q, scale
+
+
+def pack_int4(q: np.ndarray) -> np.ndarray:
+    """Storage of 4-bit codes: stored nibble u = q + 8 (1..15); every 8 consecutive elements of a
+    row form one little-endian 32-bit word whose nibble p (bits 4p..4p+3) holds element 2p and
+    whose nibble 4+p holds element 2p+1, p = 0..3.  q: int8 [m, n], n % 8 == 0.  Returns uint8
+    [m, n/2] (the words' bytes in memory order)."""
+    q = np.asarray(q, dtype=np.int8)
+    m, n = q.shape
+    if n % 8:
+        raise ValueError("n must be a multiple of 8")
+    u = (q.astype(np.int32) + 8).astype(np.uint32).reshape(m, n // 8, 8)
+    words = np.zeros((m, n // 8), dtype=np.uint32)
+    for p in range(4):
+        words |= u[:, :, 2 * p] << np.uint32(4 * p)
+        words |= u[:, :, 2 * p + 1] << np.uint32(16 + 4 * p)
+    return words.astype("<u4").view(np.uint8).reshape(m, n // 2)
+
+
+def unpack_int4(packed: np.ndarray) -> np.ndarray:
+    """Inverse of pack_int4: uint8 [m, n/2] -> int8 [m, n]."""
+    packed = np.ascontiguousarray(packed, dtype=np.uint8)
+    m, nb = packed.shape
+    words = packed.view("<u4").astype(np.uint32)
+    q = np.zeros((m, nb // 4, 8), dtype=np.int32)
+    for p in range(4):
+        q[:, :, 2 * p] = ((words >> np.uint32(4 * p)) & np.uint32(15)).astype(np.int32) - 8
+        q[:, :, 2 * p + 1] = ((words >> np.uint32(16 + 4 * p)) & np.uint32(15)).astype(np.int32) - 8
+    return q.reshape(m, nb * 2).astype(np.int8)
+
+
+def rtn_dequant(q: np.ndarray, scale: np.ndarray) -> np.ndarray:
+    """The weights a weight-only quantized linear multiplies by: scale_r * q[r, j], in fp64."""
+    return np.asarray(scale, dtype=np.float64)[:, None] * np.asarray(q, dtype=np.float64)
+
+
+def shared_ffn_rtn(x_bf16, gate, up, down) -> np.ndarray:
+    """FFN(x) of Eq. 2 with RTN weight-only quantized matrices: each of gate, up, down is a pair
+    (q int8, scale f32[rows]); activations stay bf16 values; fp64 throughout, no intermediate
+    rounding."""
+    x = bf16_to_f32(x_bf16).astype(np.float64)
+    g = x @ rtn_dequant(*gate).T
+    u = x @ rtn_dequant(*up).T
+    h = u * (g / (1.0 + np.exp(-g)))
+    return h @ rtn_dequant(*down).T
+
+
+def quantize_shared(layer: dict, bits: int) -> dict:
+    """Copy of `layer` whose shared expert is RTN-quantized to `bits` bits (Section 4.3): adds
+    layer["sh_rtn"] = {"bits", "gate": (q, scale), "up": ..., "down": ...}."""
+    out = dict(layer)
+    out["sh_rtn"] = {"bits": bits}
+    for name in ("gate", "up", "down"):
+        out["sh_rtn"][name] = rtn_quantize(bf16_to_f32(layer["sh_" + name]), bits)
+    return out
+
+
+# --------------------------------------------------------------------------------------------
 # Eq. 1-2  LN in front of the layer: RMS normalisation with unit gain (Qwen2.5's norm)
 # --------------------------------------------------------------------------------------------
 
@@ -312,7 +394,8 @@ def moe_forward(layer: dict, x_bf16: np.ndarray, residual_bf16=None, token_subse
 
     layer: dict with d, f, E, k, norm_topk, Wr[E,d] f32, router_bias[E] f32 or None,
       codes_gate/up [E][f,d] int8, codes_down [E][d,f] int8, alpha_gate/up/down f32[E],
-      sh_gate/sh_up [f,d] uint16, sh_down [d,f] uint16.
+      sh_gate/sh_up [f,d] uint16, sh_down [d,f] uint16; optional sh_rtn (see quantize_shared):
+      the shared expert then runs on its RTN-quantized weights (Section 4.3).
     token_subset: optional sorted int array; if given, the expert and shared stages are
       evaluated for those tokens only (tokens are independent of each other), while routing and
       dispatch are still computed for every token.  Row-indexed results are then in the order
@@ -364,7 +447,11 @@ def moe_forward(layer: dict, x_bf16: np.ndarray, residual_bf16=None, token_subse
         acc_gate[m] = res["acc_gate"]; acc_up[m] = res["acc_up"]; h_bf16[m] = res["h_bf16"]
         qh[m] = res["qh"]; beta_h[m] = res["beta_h"]; acc_down[m] = res["acc_down"]; y[m] = res["y"]
 
-    shared = shared_ffn(x_bf16[toks], layer["sh_gate"], layer["sh_up"], layer["sh_down"])
+    if layer.get("sh_rtn"):
+        rtn = layer["sh_rtn"]
+        shared = shared_ffn_rtn(x_bf16[toks], rtn["gate"], rtn["up"], rtn["down"])
+    else:
+        shared = shared_ffn(x_bf16[toks], layer["sh_gate"], layer["sh_up"], layer["sh_down"])
     out = shared.copy()
     if residual_bf16 is not None:
         out += bf16_to_f32(residual_bf16[toks]).astype(np.float64)

@@ -187,3 +187,46 @@ def test_workload_generators_are_seeded():
     x2 = O.bf16_to_f32(synth.tokens(synth.WORKLOADS["c2"], T=512)).astype(np.float64)
     big = (x2.std(axis=0) > 10).sum()
     assert big == 9                                                  # round(0.01 * 896)
+
+
+# ------------------------------------------------------------------ Section 4.3: RTN shared expert
+@pytest.mark.parametrize("bits", [8, 4])
+def test_rtn_layer_equals_plain_layer_when_rtn_is_lossless(bits):
+    # shared weights that already sit on the RTN grid (integers up to qmax times a power of two per
+    # row, qmax attained): quantization changes nothing, so the layer must equal the bf16 layer
+    wl, master, _, x = _tiny_layer(seed=31, d=32, f=64, E=3, k=2, T=6)
+    rng = np.random.default_rng(70 + bits)
+    qmax = 2 ** (bits - 1) - 1
+    for name, shape in (("sh_gate", (64, 32)), ("sh_up", (64, 32)), ("sh_down", (32, 64))):
+        Wi = rng.integers(-qmax, qmax + 1, size=shape)
+        Wi[:, 0] = qmax
+        row_scale = 2.0 ** rng.integers(-9, -5, size=(shape[0], 1))
+        master[name] = _bf16(Wi * row_scale)
+        assert np.array_equal(O.bf16_to_f32(master[name]).astype(np.float64), Wi * row_scale)
+    layer = O.build_layer(master)
+    plain = O.moe_forward(layer, x)
+    rtn = O.moe_forward(O.quantize_shared(layer, bits), x)
+    assert np.allclose(rtn["shared_out"], plain["shared_out"], rtol=1e-12, atol=0)
+    assert np.allclose(rtn["out"], plain["out"], rtol=1e-12, atol=0)
+
+
+@pytest.mark.parametrize("bits", [8, 4])
+def test_rtn_shared_ffn_brute_force_and_error_scale(bits):
+    wl, master, layer, x = _tiny_layer(seed=32, d=16, f=32, E=2, k=1, T=3)
+    ql = O.quantize_shared(layer, bits)
+    (qg, sg), (qu, su), (qd, sd) = (ql["sh_rtn"][n] for n in ("gate", "up", "down"))
+    xf = O.bf16_to_f32(x).astype(np.float64)
+    got = O.shared_ffn_rtn(x, (qg, sg), (qu, su), (qd, sd))
+    for t in range(3):
+        h = []
+        for r in range(32):
+            g = sum(float(sg[r]) * int(qg[r, j]) * xf[t, j] for j in range(16))
+            u = sum(float(su[r]) * int(qu[r, j]) * xf[t, j] for j in range(16))
+            h.append(u * g / (1.0 + math.exp(-g)))
+        for c in range(16):
+            ref = sum(float(sd[c]) * int(qd[c, r]) * h[r] for r in range(32))
+            assert math.isclose(got[t, c], ref, rel_tol=1e-10, abs_tol=1e-15)
+    # the quantized FFN approaches the bf16 FFN as the grid refines: INT8 error far below INT4 error
+    plain = O.shared_ffn(x, layer["sh_gate"], layer["sh_up"], layer["sh_down"])
+    rel = np.linalg.norm(got - plain) / np.linalg.norm(plain)
+    assert rel < (0.05 if bits == 8 else 0.6)

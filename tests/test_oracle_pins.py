@@ -276,3 +276,80 @@ def test_rms_norm_against_library_and_invariants():
     assert abs(r[0, 5] + 8.0) < 1e-12 and np.count_nonzero(r) == 1
     # all-zero row stays zero when eps > 0
     assert np.all(O.rms_norm(np.zeros((1, 16), np.uint16), 1e-6) == 0)
+
+
+# ------------------------------------------------------------------ Section 4.3: RTN of the shared expert
+@pytest.mark.parametrize("bits", [8, 4])
+def test_rtn_invariants(bits):
+    rng = np.random.default_rng(40 + bits)
+    qmax = 2 ** (bits - 1) - 1
+    W = O.bf16_to_f32(_bf16(rng.standard_normal((37, 96)) * 0.02))
+    W[5] = 0                                           # an all-zero output row
+    q, scale = O.rtn_quantize(W, bits)
+    Wd = W.astype(np.float64)
+    assert q.dtype == np.int8 and np.abs(q.astype(int)).max() == qmax
+    nz = np.abs(Wd).max(axis=1) > 0
+    assert np.all(np.abs(q[nz].astype(int)).max(axis=1) == qmax)       # the absmax element maps to +-qmax
+    assert not q[5].any()
+    # scale = absmax / qmax, to one fp32 rounding
+    assert np.allclose(scale[nz].astype(np.float64), np.abs(Wd[nz]).max(axis=1) / qmax, rtol=2 ** -23)
+    # round-to-nearest: |w - scale*q| <= scale/2 (+ the fp32 roundings of the pinned sequence)
+    err = np.abs(Wd - O.rtn_dequant(q, scale))
+    assert np.all(err <= scale.astype(np.float64)[:, None] * (0.5 + 1e-5))
+    # odd symmetry and power-of-two scale invariance
+    qn, sn = O.rtn_quantize(-W, bits)
+    assert np.array_equal(qn, -q) and np.array_equal(sn, scale)
+    q8, s8 = O.rtn_quantize(W * np.float32(8), bits)
+    assert np.array_equal(q8, q) and np.array_equal(s8[nz], scale[nz] * 8)
+    # nearest grid point by brute force in exact rational arithmetic, away from ties
+    for r in (0, 11, 36):
+        beta = Fraction(float(np.abs(W[r]).max()))
+        for j in range(0, 96, 7):
+            t = Fraction(float(W[r, j])) * qmax / beta
+            lo = math.floor(t)
+            if abs(t - lo - Fraction(1, 2)) > Fraction(1, 1000):
+                assert int(q[r, j]) == (lo if t - lo < Fraction(1, 2) else lo + 1)
+
+
+@pytest.mark.parametrize("bits", [8, 4])
+def test_rtn_integer_rows_are_lossless(bits):
+    # rows of integers in [-qmax, qmax] (times a power of two) that attain qmax: q = the integers, scale = 2^j
+    rng = np.random.default_rng(50 + bits)
+    qmax = 2 ** (bits - 1) - 1
+    Wi = rng.integers(-qmax, qmax + 1, size=(12, 64))
+    Wi[:, 3] = qmax
+    q, scale = O.rtn_quantize((Wi * 0.25).astype(np.float32), bits)
+    assert np.array_equal(q, Wi) and np.all(scale == np.float32(0.25))
+    assert np.array_equal(O.rtn_dequant(q, scale), Wi * 0.25)
+
+
+def test_rtn_int8_is_eq8_applied_to_weight_rows():
+    # with 8 bits the quantizer is Eq. 8 with a weight row in the place of a token
+    rng = np.random.default_rng(60)
+    Wb = _bf16(rng.standard_normal((21, 80)) * 0.02)
+    q, scale = O.rtn_quantize(O.bf16_to_f32(Wb), 8)
+    qa, beta, _ = O.quant_act(Wb)
+    assert np.array_equal(q, qa) and np.array_equal(scale, beta / np.float32(127))
+
+
+def test_int4_storage_by_hand_and_size():
+    # one word by hand: elements 0..7 = -8+u with u = 1..8 -> nibbles (e0,e2,e4,e6 | e1,e3,e5,e7)
+    q = np.array([[-7, -6, -5, -4, -3, -2, -1, 0]], dtype=np.int8)
+    packed = O.pack_int4(q)
+    word = int.from_bytes(bytes(packed[0]), "little")
+    assert word == 0x8642_7531
+    # independent decoder: python integers
+    rng = np.random.default_rng(61)
+    q = rng.integers(-7, 8, size=(5, 48)).astype(np.int8)
+    packed = O.pack_int4(q)
+    assert packed.shape == (5, 24) and packed.dtype == np.uint8          # 4 bits per weight
+    for r in range(5):
+        for w in range(6):
+            word = int.from_bytes(bytes(packed[r, 4 * w:4 * w + 4]), "little")
+            for p in range(4):
+                assert ((word >> (4 * p)) & 15) - 8 == q[r, 8 * w + 2 * p]
+                assert ((word >> (16 + 4 * p)) & 15) - 8 == q[r, 8 * w + 2 * p + 1]
+    assert np.array_equal(O.unpack_int4(packed), q)
+    # bytes per weight behind the Table 3 footprints: 1 (INT8) and 1/2 (INT4), scales not counted
+    q8, _ = O.rtn_quantize(rng.standard_normal((16, 64)).astype(np.float32), 8)
+    assert q8.nbytes == 16 * 64 and packed.nbytes * 2 == q.size
