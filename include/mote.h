@@ -6,7 +6,8 @@
  *
  * FFN is the bf16 shared SwiGLU expert; FFN^T_e are routed GLU experts whose weights are ternary
  * {-1,0,1} with one absmean scale per matrix (Eq. 7, 9) and whose inputs are per-token absmax int8
- * (Eq. 8).  Ternary weights are stored as INT2 (Section 3.1, last paragraph).
+ * (Eq. 8).  Ternary weights are stored as INT2 (Section 3.1, last paragraph).  The shared expert
+ * may also be held as RTN weight-only INT8 or INT4 codes (post-training quantization, Section 4.3).
  *
  * General rules for every entry point
  *   - Pointers are DEVICE pointers unless an argument name ends in `_host`.  The caller owns all
@@ -43,6 +44,8 @@ typedef enum {
 
 enum { MOTE_DTYPE_F32 = 0, MOTE_DTYPE_BF16 = 1 };
 enum { MOTE_MAX_EXPERTS = 64, MOTE_MAX_TOPK = 8 };
+/* storage of the shared expert's three matrices (mote_layer_t.shared_bits; 0 means bf16) */
+enum { MOTE_SHARED_BF16 = 16, MOTE_SHARED_INT8 = 8, MOTE_SHARED_INT4 = 4 };
 
 /* Which implementation runs the layer.  AUTO picks per shape; the others force one path (used by
  * the tests to check every path against the oracle).
@@ -107,6 +110,32 @@ mote_status_t mote_ternarize_pack_static(const void* W, int w_dtype, int64_t m, 
                                          uint8_t* packed, float* alpha, void* stream);
 
 /* ------------------------------------------------------------------------------------------------
+ * mote_rtn_quant -- round-to-nearest absmax weight quantizer for the shared expert (Section 4.3:
+ * the shared expert is post-training quantized to INT8, or INT4 under tighter memory budgets).
+ * The paper names the method (RTN) and the bit widths only; this library takes one scale per
+ * output row, the absmax form of Eq. 8-10 applied to the rows of W.  Offline step, once per matrix.
+ *
+ *   qmax     = 2^(bits-1) - 1                                   127 or 7
+ *   beta_r   = max( max_j |W[r,j]|, 1e-5 )
+ *   q[r,j]   = clamp( rint( (qmax * W[r,j]) / beta_r ), -qmax, qmax )   fp32 multiply, true fp32
+ *                                                                division, ties to even
+ *   scale[r] = beta_r / qmax                                    dequantized weight = scale[r] * q[r,j]
+ *
+ *   W      in   [m, n] row-major, dtype w_dtype (MOTE_DTYPE_F32 or MOTE_DTYPE_BF16), 16-B aligned
+ *   bits   8 or 4
+ *   q      out  bits = 8: [m, n] int8.
+ *               bits = 4: [m, n/2] bytes; stored nibble u = q + 8 (1..15); every 8 consecutive
+ *               elements of a row form one little-endian 32-bit word whose nibble p (bits 4p..4p+3)
+ *               holds element 2p and whose nibble 4+p holds element 2p+1, p = 0..3.  (Both halves of
+ *               the word then expand to element pairs with one mask each.)
+ *               16-B aligned.
+ *   scale  out  [m] float
+ * Errors: NULL -> ERR_NULL; m<=0, n<=0, n%16 != 0, n > 65536, bits not 8 or 4 -> ERR_SHAPE; ERR_DTYPE; ERR_ALIGN.
+ */
+mote_status_t mote_rtn_quant(const void* W, int w_dtype, int64_t m, int64_t n, int bits,
+                             void* q, float* scale, void* stream);
+
+/* ------------------------------------------------------------------------------------------------
  * mote_quant_act -- per-token absmax int8 activation quantizer (Eq. 8, 9, 10).
  *
  *   beta_t = max( max_j |x[t,j]|, 1e-5 );   q[t,j] = clamp( rint( (127 * x[t,j]) / beta_t ), -128, 127 )
@@ -151,9 +180,13 @@ typedef struct {
   const float* alpha_gate;         /* [E]                                                       */
   const float* alpha_up;           /* [E]                                                       */
   const float* alpha_down;         /* [E]                                                       */
-  const void* sh_gate;             /* bf16 [f, d]  shared expert                                */
-  const void* sh_up;               /* bf16 [f, d]                                               */
-  const void* sh_down;             /* bf16 [d, f]                                               */
+  const void* sh_gate;             /* [f, d]  shared expert: bf16, or the q of mote_rtn_quant   */
+  const void* sh_up;               /* [f, d]                                                    */
+  const void* sh_down;             /* [d, f]                                                    */
+  int32_t shared_bits;             /* MOTE_SHARED_BF16 (or 0), MOTE_SHARED_INT8, MOTE_SHARED_INT4 */
+  const float* sh_gate_scale;      /* [f]  scales of mote_rtn_quant when shared_bits is 8 or 4,  */
+  const float* sh_up_scale;        /* [f]  16-B aligned; ignored for bf16                        */
+  const float* sh_down_scale;      /* [d]                                                       */
 } mote_layer_t;
 
 /* Optional copies of intermediates (for parity checks).  Every member may be NULL; a non-NULL
@@ -182,6 +215,9 @@ size_t mote_workspace_bytes(int d, int f, int E, int k, int64_t T_max);
  * mote_moe_forward -- the whole layer (Eq. 2-8): route, dispatch, Q_a(x), gate/up ternary GEMM
  * with fused dequantisation and SwiGLU, Q_a(h), down ternary GEMM, shared bf16 FFN, gate-weighted
  * combine with the shared output and the optional residual.
+ * With shared_bits 8 or 4 the shared FFN is weight-only quantized (Section 4.3): its activations
+ * (x, and h rounded to bf16) stay bf16, the integer codes enter the bf16 tensor-core MMAs exactly
+ * (|q| <= 127 is representable), accumulation is fp32 and the row scale multiplies the finished sum.
  *
  *   x_bf16         in   [T, d] bf16 contiguous, 16-B aligned
  *   residual_bf16  in   [T, d] bf16 or NULL; may alias out_bf16

@@ -24,7 +24,9 @@ class mote_layer_t(C.Structure):
                 ("Wr", C.c_void_p), ("router_bias", C.c_void_p),
                 ("gate_packed", C.c_void_p), ("up_packed", C.c_void_p), ("down_packed", C.c_void_p),
                 ("alpha_gate", C.c_void_p), ("alpha_up", C.c_void_p), ("alpha_down", C.c_void_p),
-                ("sh_gate", C.c_void_p), ("sh_up", C.c_void_p), ("sh_down", C.c_void_p)]
+                ("sh_gate", C.c_void_p), ("sh_up", C.c_void_p), ("sh_down", C.c_void_p),
+                ("shared_bits", C.c_int32),
+                ("sh_gate_scale", C.c_void_p), ("sh_up_scale", C.c_void_p), ("sh_down_scale", C.c_void_p)]
 
 
 TAP_FIELDS = ["topk_idx", "topk_w", "offsets", "perm", "qx", "beta_x", "acc_gate", "acc_up", "h_bf16",
@@ -45,6 +47,8 @@ lib.mote_ternarize_pack.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int64, C
 lib.mote_ternarize_pack_static.restype = C.c_int
 lib.mote_ternarize_pack_static.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p,
                                            C.c_void_p]
+lib.mote_rtn_quant.restype = C.c_int
+lib.mote_rtn_quant.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int64, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
 lib.mote_quant_act.restype = C.c_int
 lib.mote_quant_act.argtypes = [C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p,
                                C.c_void_p, C.c_void_p]
@@ -131,6 +135,21 @@ def mote_ternarize_pack_static(W: torch.Tensor, packed: torch.Tensor, alpha: tor
     return packed, alpha
 
 
+def mote_rtn_quant(W: torch.Tensor, bits: int):
+    """Section 4.3: RTN absmax codes of W[m, n] (fp32 or bf16, CUDA), one scale per row.
+    Returns (q, scale float32[m]); q is int8[m, n] for bits = 8 and uint8[m, n/2] for bits = 4."""
+    _need_cuda(W)
+    m, n = W.shape
+    dt = {torch.float32: DTYPE_F32, torch.bfloat16: DTYPE_BF16}[W.dtype]
+    if bits == 8:
+        q = torch.empty((m, n), dtype=torch.int8, device=W.device)
+    else:
+        q = torch.empty((m, max(n // 2, 1)), dtype=torch.uint8, device=W.device)
+    scale = torch.empty(m, dtype=torch.float32, device=W.device)
+    _check(lib.mote_rtn_quant(_ptr(W), dt, m, n, bits, _ptr(q), _ptr(scale), _stream()), "mote_rtn_quant")
+    return q, scale
+
+
 def mote_quant_act(x: torch.Tensor, want_rowsum: bool = True):
     """Eq. 8: x[T, d] bf16 (CUDA; rows may be strided) -> (q int8[T,d], beta f32[T], rowsum i32[T])."""
     if not x.is_cuda or x.dtype != torch.bfloat16 or x.stride(1) != 1:
@@ -161,11 +180,14 @@ class MoteLayer:
     """Device-resident weights of one MoTE layer plus its mote_layer_t."""
 
     def __init__(self, d, f, E, k, norm_topk, Wr, router_bias, gate_packed, up_packed, down_packed,
-                 alpha_gate, alpha_up, alpha_down, sh_gate, sh_up, sh_down, path=PATH_AUTO):
+                 alpha_gate, alpha_up, alpha_down, sh_gate, sh_up, sh_down, path=PATH_AUTO,
+                 shared_bits=16, sh_gate_scale=None, sh_up_scale=None, sh_down_scale=None):
         self.d, self.f, self.E, self.k, self.norm_topk, self.path = d, f, E, k, norm_topk, path
+        self.shared_bits = shared_bits
         self.tensors = dict(Wr=Wr, router_bias=router_bias, gate_packed=gate_packed, up_packed=up_packed,
                             down_packed=down_packed, alpha_gate=alpha_gate, alpha_up=alpha_up,
-                            alpha_down=alpha_down, sh_gate=sh_gate, sh_up=sh_up, sh_down=sh_down)
+                            alpha_down=alpha_down, sh_gate=sh_gate, sh_up=sh_up, sh_down=sh_down,
+                            sh_gate_scale=sh_gate_scale, sh_up_scale=sh_up_scale, sh_down_scale=sh_down_scale)
         _need_cuda(*self.tensors.values())
         self._ws = None
 
@@ -215,12 +237,24 @@ class MoteLayer:
                    packed["gate"], packed["up"], packed["down"], alphas["gate"], alphas["up"], alphas["down"],
                    draw("sh_gate").contiguous(), draw("sh_up").contiguous(), draw("sh_down").contiguous(), path=path)
 
+    def quantize_shared(self, bits: int, path=None) -> "MoteLayer":
+        """Section 4.3: a layer with the same routed experts whose (bf16) shared expert is replaced
+        by its RTN INT8 / INT4 codes (mote_rtn_quant on the device)."""
+        if self.shared_bits != 16:
+            raise ValueError("the shared expert is quantized already")
+        t = dict(self.tensors)
+        for name in ("sh_gate", "sh_up", "sh_down"):
+            t[name], t[name + "_scale"] = mote_rtn_quant(self.tensors[name], bits)
+        return MoteLayer(self.d, self.f, self.E, self.k, self.norm_topk, path=self.path if path is None else path,
+                         shared_bits=bits, **t)
+
     def struct(self) -> mote_layer_t:
         t = self.tensors
         s = mote_layer_t(self.d, self.f, self.E, self.k, self.norm_topk, self.path)
         for name in ("Wr", "router_bias", "gate_packed", "up_packed", "down_packed", "alpha_gate", "alpha_up",
-                     "alpha_down", "sh_gate", "sh_up", "sh_down"):
+                     "alpha_down", "sh_gate", "sh_up", "sh_down", "sh_gate_scale", "sh_up_scale", "sh_down_scale"):
             setattr(s, name, None if t[name] is None else t[name].data_ptr())
+        s.shared_bits = self.shared_bits
         return s
 
     def workspace(self, T: int, host_staging: bool = False) -> torch.Tensor:

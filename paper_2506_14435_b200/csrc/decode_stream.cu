@@ -6,7 +6,8 @@
 // never stage weights in shared memory: each lane loads 16 bytes of one weight row straight from
 // global memory into registers, expands the 2-bit codes there (one shift and one mask per four
 // codes) and feeds them to warp-level tensor-core MMAs (mma.sync m16n8k32 u8 x s8 -> s32 for the
-// ternary experts, m16n8k16 bf16 for the shared expert) as the A operand, with the tokens as the
+// ternary experts, m16n8k16 bf16 for the shared expert -- whose weights are bf16, or RTN INT8/INT4
+// codes (Section 4.3) expanded to bf16 in registers) as the A operand, with the tokens as the
 // 8-wide B operand.  The reduction index of an integer dot product can be permuted freely, so a
 // lane's 64 consecutive codes need no shuffling: the token operand is stored in the matching
 // ("k-interleaved") order by the quantizer.
@@ -362,11 +363,96 @@ __device__ __forceinline__ void bf16_rows_steps(const uint16_t* __restrict__ row
   }
 }
 
+// RTN-coded rows (Section 4.3): one step covers 64 bytes of each row (64 int8 or 128 4-bit codes):
+// lane (g, t) loads bytes [64*step + 16*t, +16) of row A and row B, expands them to bf16 pairs in
+// registers and multiplies them with the same elements of its token column.  A lane past the end
+// of a short last step contributes zeros.
+template <int NT, int kBits>
+__device__ __forceinline__ void rtn_rows_steps(const uint8_t* __restrict__ row_a, const uint8_t* __restrict__ row_b,
+                                               const uint16_t* const (&tok)[NT], int step_begin, int step_end,
+                                               int k_bytes, int lane, float (&acc)[NT][4]) {
+  constexpr int kElems = kBits == 8 ? 16 : 32;        // elements in 16 bytes
+  const int t = lane & 3;
+  const uint32_t z = kBits == 8 ? 0u : 0x88888888u;   // codes of weight 0
+  const uint4 kZero = make_uint4(z, z, z, z);
+  uint4 qa[kBf16Ahead], qb[kBf16Ahead];
+#pragma unroll
+  for (int i = 0; i < kBf16Ahead; ++i) {
+    const int off = (step_begin + i) * 64 + t * 16;
+    const bool ok = step_begin + i < step_end && off < k_bytes;
+    qa[i] = ok ? ldg_stream16(row_a + off) : kZero;
+    qb[i] = ok ? ldg_stream16(row_b + off) : kZero;
+  }
+  for (int s0 = step_begin; s0 < step_end; s0 += kBf16Ahead) {
+#pragma unroll
+    for (int i = 0; i < kBf16Ahead; ++i) {
+      const int s = s0 + i;
+      if (s < step_end) {
+        const uint32_t wa[4] = {qa[i].x, qa[i].y, qa[i].z, qa[i].w};
+        const uint32_t wb[4] = {qb[i].x, qb[i].y, qb[i].z, qb[i].w};
+        {
+          const int off = (s + kBf16Ahead) * 64 + t * 16;
+          const bool ok = s + kBf16Ahead < step_end && off < k_bytes;
+          qa[i] = ok ? ldg_stream16(row_a + off) : kZero;
+          qb[i] = ok ? ldg_stream16(row_b + off) : kZero;
+        }
+        const bool q_ok = (s * 64 + t * 16) < k_bytes;
+        const int e0 = (s * 4 + t) * kElems;          // first element of this lane's 16 bytes
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {
+          if (kBits == 8) {
+            uint32_t a01, a23, b01, b23;
+            s8x4_to_bf16x2(wa[w], a01, a23);
+            s8x4_to_bf16x2(wb[w], b01, b23);
+#pragma unroll
+            for (int n = 0; n < NT; ++n) {
+              uint2 q = make_uint2(0u, 0u);
+              if (tok[n] && q_ok) q = *reinterpret_cast<const uint2*>(tok[n] + e0 + 4 * w);
+              mma_bf16(acc[n], a01, b01, a23, b23, q.x, q.y);
+            }
+          } else {
+            uint32_t ea[4], eb[4];
+            u4x8_to_bf16x2(wa[w], ea);
+            u4x8_to_bf16x2(wb[w], eb);
+#pragma unroll
+            for (int n = 0; n < NT; ++n) {
+              uint4 q = make_uint4(0u, 0u, 0u, 0u);
+              if (tok[n] && q_ok) q = *reinterpret_cast<const uint4*>(tok[n] + e0 + 8 * w);
+              mma_bf16(acc[n], ea[0], eb[0], ea[1], eb[1], q.x, q.y);
+              mma_bf16(acc[n], ea[2], eb[2], ea[3], eb[3], q.z, q.w);
+            }
+          }
+        }
+      }
+    }
+  }
+}
+
 // splits n_steps as evenly as possible over n_parts; part p gets [begin, end)
 __device__ __forceinline__ void split_steps(int n_steps, int n_parts, int p, int& begin, int& end) {
   const int base = n_steps / n_parts, rem = n_steps % n_parts;
   begin = p * base + min(p, rem);
   end = begin + base + (p < rem ? 1 : 0);
+}
+
+// Two rows of one shared-expert matrix against the token columns: bf16 values or RTN codes.
+// K = reduction length in elements; warp `part` of `n_parts` takes its share of the steps.
+template <int NT>
+__device__ __forceinline__ void shared_rows(const void* W, int bits, int64_t row_a, int64_t row_b, int K,
+                                            const uint16_t* const (&tok)[NT], int n_parts, int part, int lane,
+                                            float (&acc)[NT][4]) {
+  int sb, se;
+  if (bits == 16) {
+    const uint16_t* w = static_cast<const uint16_t*>(W);
+    split_steps(K / 32, n_parts, part, sb, se);
+    bf16_rows_steps<NT>(w + row_a * K, w + row_b * K, tok, sb, se, lane, acc);
+  } else {
+    const uint8_t* w = static_cast<const uint8_t*>(W);
+    const int k_bytes = bits == 8 ? K : K / 2;
+    split_steps((k_bytes + 63) / 64, n_parts, part, sb, se);
+    if (bits == 8) rtn_rows_steps<NT, 8>(w + row_a * k_bytes, w + row_b * k_bytes, tok, sb, se, k_bytes, lane, acc);
+    else rtn_rows_steps<NT, 4>(w + row_a * k_bytes, w + row_b * k_bytes, tok, sb, se, k_bytes, lane, acc);
+  }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -410,7 +496,7 @@ struct DecodeGateUpArgs {
   DecodeCommon c;
   const uint8_t* gate_packed; const uint8_t* up_packed;   // [E][f, d/4]
   const float* alpha_gate; const float* alpha_up;
-  const uint16_t* sh_gate; const uint16_t* sh_up;          // [f, d] bf16
+  SharedMat sh_gate, sh_up; int sh_bits;                   // [f, d] bf16, or RTN codes + row scales
   const uint16_t* x;                                       // [T, d] bf16
   uint16_t* h;              // [P, f] bf16, sorted rows
   uint32_t* beta_h_bits;    // [P]
@@ -485,15 +571,29 @@ __device__ __forceinline__ void gateup_shared_tile(const DecodeGateUpArgs& a, in
   float acc[NT][4];
 #pragma unroll
   for (int n = 0; n < NT; ++n) acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.0f;
-  int sb, se;
-  split_steps(d / 32, kGuWarps, warp, sb, se);
-  bf16_rows_steps<NT>(a.sh_gate + int64_t(frow) * d, a.sh_up + int64_t(frow) * d, tok, sb, se, lane, acc);
+  // gate row in fragment rows 0-7, up row in 8-15: two different matrices, one call each half
+  if (a.sh_bits == 16) {
+    int sb, se;
+    split_steps(d / 32, kGuWarps, warp, sb, se);
+    bf16_rows_steps<NT>(static_cast<const uint16_t*>(a.sh_gate.w) + int64_t(frow) * d,
+                        static_cast<const uint16_t*>(a.sh_up.w) + int64_t(frow) * d, tok, sb, se, lane, acc);
+  } else {
+    const int k_bytes = a.sh_bits == 8 ? d : d / 2;
+    const uint8_t* rg = static_cast<const uint8_t*>(a.sh_gate.w) + int64_t(frow) * k_bytes;
+    const uint8_t* ru = static_cast<const uint8_t*>(a.sh_up.w) + int64_t(frow) * k_bytes;
+    int sb, se;
+    split_steps((k_bytes + 63) / 64, kGuWarps, warp, sb, se);
+    if (a.sh_bits == 8) rtn_rows_steps<NT, 8>(rg, ru, tok, sb, se, k_bytes, lane, acc);
+    else rtn_rows_steps<NT, 4>(rg, ru, tok, sb, se, k_bytes, lane, acc);
+  }
   // partial sums of the 4 warps are added in warp order
 #pragma unroll
   for (int n = 0; n < NT; ++n)
 #pragma unroll
     for (int i = 0; i < 4; ++i) s_part[(warp * NT * 4 + n * 4 + i) * 32 + lane] = acc[n][i];
   __syncthreads();
+  const float sc_g = a.sh_bits == 16 ? 1.0f : a.sh_gate.scale[frow];
+  const float sc_u = a.sh_bits == 16 ? 1.0f : a.sh_up.scale[frow];
   for (int n = warp; n < NT; n += kGuWarps) {
     float v[4];
 #pragma unroll
@@ -507,7 +607,7 @@ __device__ __forceinline__ void gateup_shared_tile(const DecodeGateUpArgs& a, in
     for (int j = 0; j < 2; ++j) {
       const int token = n * 8 + 2 * t + j;
       if (token < T) {
-        const float gv = v[j], uv = v[2 + j];
+        const float gv = v[j] * sc_g, uv = v[2 + j] * sc_u;
         const float hv = uv * __fdividef(gv, 1.0f + __expf(-gv));
         a.hs[int64_t(token) * f + frow] = (uint16_t)f32_to_bf16_bits(hv);
       }
@@ -562,7 +662,7 @@ struct DecodeDownArgs {
   DecodeCommon c;
   const uint8_t* down_packed;   // [E][d, f/4]
   const float* alpha_down;
-  const uint16_t* sh_down;      // [d, f] bf16
+  SharedMat sh_down; int sh_bits;   // [d, f] bf16, or RTN codes + row scales
   const int8_t* qh;             // [P, f] sorted rows, k-interleaved
   const float* beta_h;          // [P]
   const int32_t* rowsum_h;      // [P]
@@ -640,14 +740,14 @@ __device__ __forceinline__ void down_shared_tile(const DecodeDownArgs& a, int ti
   float acc[NT][4];
 #pragma unroll
   for (int n = 0; n < NT; ++n) acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.0f;
-  int sb, se;
-  split_steps(f / 32, kDownWarps, warp, sb, se);
-  bf16_rows_steps<NT>(a.sh_down + int64_t(drow) * f, a.sh_down + int64_t(drow + 8) * f, tok, sb, se, lane, acc);
+  shared_rows<NT>(a.sh_down.w, a.sh_bits, drow, drow + 8, f, tok, kDownWarps, warp, lane, acc);
 #pragma unroll
   for (int n = 0; n < NT; ++n)
 #pragma unroll
     for (int i = 0; i < 4; ++i) s_part[(warp * NT * 4 + n * 4 + i) * 32 + lane] = acc[n][i];
   __syncthreads();
+  const float sc_lo = a.sh_bits == 16 ? 1.0f : a.sh_down.scale[drow];
+  const float sc_hi = a.sh_bits == 16 ? 1.0f : a.sh_down.scale[drow + 8];
   for (int n = warp; n < NT; n += kDownWarps) {
     float v[4];
 #pragma unroll
@@ -661,8 +761,8 @@ __device__ __forceinline__ void down_shared_tile(const DecodeDownArgs& a, int ti
     for (int j = 0; j < 2; ++j) {
       const int token = n * 8 + 2 * t + j;
       if (token < T) {
-        a.s[int64_t(token) * d + drow] = v[j];
-        a.s[int64_t(token) * d + drow + 8] = v[2 + j];
+        a.s[int64_t(token) * d + drow] = v[j] * sc_lo;
+        a.s[int64_t(token) * d + drow + 8] = v[2 + j] * sc_hi;
       }
     }
   }
@@ -750,8 +850,8 @@ mote_status_t launch_decode_stream(const DecodeStreamArgs& p, int phase, cudaStr
   if (phase == 1) {
     DecodeGateUpArgs ga{};
     ga.c = c; ga.gate_packed = p.gate_packed; ga.up_packed = p.up_packed; ga.alpha_gate = p.alpha_gate;
-    ga.alpha_up = p.alpha_up; ga.sh_gate = static_cast<const uint16_t*>(p.sh_gate);
-    ga.sh_up = static_cast<const uint16_t*>(p.sh_up); ga.x = static_cast<const uint16_t*>(p.x);
+    ga.alpha_up = p.alpha_up; ga.sh_gate = p.sh_gate;
+    ga.sh_up = p.sh_up; ga.sh_bits = p.shared_bits; ga.x = static_cast<const uint16_t*>(p.x);
     ga.h = static_cast<uint16_t*>(p.h); ga.beta_h_bits = reinterpret_cast<uint32_t*>(p.beta_h);
     ga.hs = static_cast<uint16_t*>(p.hs); ga.tap_gate = p.tap_gate; ga.tap_up = p.tap_up;
     const int tiles = f / 8, quads = (tiles + kGuWarps - 1) / kGuWarps;
@@ -768,7 +868,7 @@ mote_status_t launch_decode_stream(const DecodeStreamArgs& p, int phase, cudaStr
 
   DecodeDownArgs da{};
   da.c = c; da.down_packed = p.down_packed; da.alpha_down = p.alpha_down;
-  da.sh_down = static_cast<const uint16_t*>(p.sh_down); da.qh = p.qh; da.beta_h = p.beta_h; da.rowsum_h = p.rowsum_h;
+  da.sh_down = p.sh_down; da.sh_bits = p.shared_bits; da.qh = p.qh; da.beta_h = p.beta_h; da.rowsum_h = p.rowsum_h;
   da.hs = static_cast<const uint16_t*>(p.hs); da.y = p.y; da.s = p.s; da.tap_down = p.tap_down;
   const int tiles = d / 16;
   const int max_items = tiles + std::min<int>(E, T * k) * tiles;

@@ -4,7 +4,7 @@
 //   ternary gate/up (Eq. 6):  acc_g, acc_u = codes . q  (dp4a, exact int32)
 //                             h = bf16(u * silu(g)),  g = fl32(acc_g)*alpha_g*(beta/127), u likewise
 //   ternary down    (Eq. 5):  y = fl32(acc_d) * alpha_d*(beta_h/127)
-//   shared gate/up, down (Eq. 2): bf16 operands, fp32 FMA accumulation
+//   shared gate/up, down (Eq. 2): bf16 operands (or RTN codes, Section 4.3), fp32 FMA accumulation
 //
 // Rows are in expert-sorted order; a CTA owns a 32-row x 64-column tile of one expert.
 #include "mote_common.cuh"
@@ -150,10 +150,36 @@ mote_status_t launch_ternary_down_simt(const TernaryGemmArgs& a, cudaStream_t s)
 // ---------------------------------------------------------------------------------------------
 constexpr int kSK = 32;      // reduction elements per step (bf16 path)
 
-template <bool kGateUp>
+// kBits: 16 = bf16 weights; 8 / 4 = RTN codes (Section 4.3), expanded here and scaled per output
+// column after the sum.
+template <int kBits>
+__device__ __forceinline__ void load_w8(const void* W, int64_t row, int K, int k, float (&v)[8]) {
+  if (kBits == 16) {
+    const uint4 r = *reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(W) + row * K + k);
+    const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) { v[2 * j] = bf16_lo(w[j]); v[2 * j + 1] = bf16_hi(w[j]); }
+  } else if (kBits == 8) {
+    const uint2 r = *reinterpret_cast<const uint2*>(static_cast<const int8_t*>(W) + row * K + k);
+    const uint32_t w[2] = {r.x, r.y};
+#pragma unroll
+    for (int j = 0; j < 8; ++j) v[j] = (float)(int8_t)((w[j >> 2] >> (8 * (j & 3))) & 0xFFu);
+  } else {
+    const uint32_t word = *reinterpret_cast<const uint32_t*>(static_cast<const uint8_t*>(W) + row * (K / 2) + k / 2);
+#pragma unroll
+    for (int p = 0; p < 4; ++p) {
+      v[2 * p] = (float)((int)((word >> (4 * p)) & 15u) - 8);
+      v[2 * p + 1] = (float)((int)((word >> (16 + 4 * p)) & 15u) - 8);
+    }
+  }
+}
+
+template <bool kGateUp, int kBits>
 __global__ void __launch_bounds__(256) shared_gemm_simt_kernel(const uint16_t* __restrict__ A, int64_t M, int K,
-                                                               const uint16_t* __restrict__ W0,
-                                                               const uint16_t* __restrict__ W1, int N,
+                                                               const void* __restrict__ W0,
+                                                               const void* __restrict__ W1,
+                                                               const float* __restrict__ scale0,
+                                                               const float* __restrict__ scale1, int N,
                                                                uint16_t* __restrict__ h_out,
                                                                float* __restrict__ s_out) {
   constexpr int kMats = kGateUp ? 2 : 1;
@@ -185,12 +211,10 @@ __global__ void __launch_bounds__(256) shared_gemm_simt_kernel(const uint16_t* _
     for (int i = tid; i < kMats * kTN * 4; i += 256) {
       const int wr = i >> 2, u = i & 3;
       const int m = wr / kTN, c = wr % kTN;
-      uint4 v = make_uint4(0, 0, 0, 0);
-      if (col0 + c < N && k0 + u * 8 < K)
-        v = *reinterpret_cast<const uint4*>((m == 0 ? W0 : W1) + int64_t(col0 + c) * K + k0 + u * 8);
-      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+      float v[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+      if (col0 + c < N && k0 + u * 8 < K) load_w8<kBits>(m == 0 ? W0 : W1, col0 + c, K, k0 + u * 8, v);
 #pragma unroll
-      for (int j = 0; j < 4; ++j) { Bs[wr][u * 8 + 2 * j] = bf16_lo(w[j]); Bs[wr][u * 8 + 2 * j + 1] = bf16_hi(w[j]); }
+      for (int j = 0; j < 8; ++j) Bs[wr][u * 8 + j] = v[j];
     }
     __syncthreads();
 #pragma unroll 8
@@ -215,35 +239,45 @@ __global__ void __launch_bounds__(256) shared_gemm_simt_kernel(const uint16_t* _
     for (int c = 0; c < 4; ++c) {
       const int col = col0 + tx + 16 * c;
       if (col >= N) continue;
+      const float s0 = kBits == 16 ? 1.0f : scale0[col];
       if (kGateUp) {
-        const float g = acc[0][r][c], u = acc[1][r][c];
+        const float s1 = kBits == 16 ? 1.0f : scale1[col];
+        const float g = acc[0][r][c] * s0, u = acc[1][r][c] * s1;
         const float h = u * (g / (1.0f + expf(-g)));
         h_out[row * N + col] = (uint16_t)f32_to_bf16_bits(h);
       } else {
-        s_out[row * N + col] = acc[0][r][c];
+        s_out[row * N + col] = acc[0][r][c] * s0;
       }
     }
   }
 }
 
-mote_status_t launch_shared_gateup_simt(const void* x, const void* Wg, const void* Wu, int64_t T, int d, int f,
-                                        void* h_bf16, cudaStream_t stream) {
+template <bool kGateUp>
+static void launch_shared_simt(dim3 grid, cudaStream_t stream, int bits, const uint16_t* A, int64_t M, int K,
+                               const void* W0, const void* W1, const float* s0, const float* s1, int N,
+                               uint16_t* h_out, float* s_out) {
+  if (bits == 8) shared_gemm_simt_kernel<kGateUp, 8><<<grid, 256, 0, stream>>>(A, M, K, W0, W1, s0, s1, N, h_out, s_out);
+  else if (bits == 4) shared_gemm_simt_kernel<kGateUp, 4><<<grid, 256, 0, stream>>>(A, M, K, W0, W1, s0, s1, N, h_out, s_out);
+  else shared_gemm_simt_kernel<kGateUp, 16><<<grid, 256, 0, stream>>>(A, M, K, W0, W1, s0, s1, N, h_out, s_out);
+}
+
+mote_status_t launch_shared_gateup_simt(const void* x, const SharedMat& Wg, const SharedMat& Wu, int bits, int64_t T,
+                                        int d, int f, void* h_bf16, cudaStream_t stream) {
   if (T == 0) return MOTE_OK;
   dim3 grid((f + kTN - 1) / kTN, (unsigned)((T + kTM - 1) / kTM));
-  shared_gemm_simt_kernel<true><<<grid, 256, 0, stream>>>(
-      static_cast<const uint16_t*>(x), T, d, static_cast<const uint16_t*>(Wg), static_cast<const uint16_t*>(Wu),
-      f, static_cast<uint16_t*>(h_bf16), nullptr);
+  launch_shared_simt<true>(grid, stream, bits, static_cast<const uint16_t*>(x), T, d, Wg.w, Wu.w, Wg.scale, Wu.scale,
+                           f, static_cast<uint16_t*>(h_bf16), nullptr);
   ++g_launch_count;
   MOTE_LAUNCH_OK();
   return MOTE_OK;
 }
 
-mote_status_t launch_shared_down_simt(const void* h, const void* Wd, int64_t T, int d, int f, float* s,
+mote_status_t launch_shared_down_simt(const void* h, const SharedMat& Wd, int bits, int64_t T, int d, int f, float* s,
                                       cudaStream_t stream) {
   if (T == 0) return MOTE_OK;
   dim3 grid((d + kTN - 1) / kTN, (unsigned)((T + kTM - 1) / kTM));
-  shared_gemm_simt_kernel<false><<<grid, 256, 0, stream>>>(static_cast<const uint16_t*>(h), T, f,
-                                                           static_cast<const uint16_t*>(Wd), nullptr, d, nullptr, s);
+  launch_shared_simt<false>(grid, stream, bits, static_cast<const uint16_t*>(h), T, f, Wd.w, nullptr, Wd.scale, nullptr,
+                            d, nullptr, s);
   ++g_launch_count;
   MOTE_LAUNCH_OK();
   return MOTE_OK;

@@ -151,8 +151,15 @@ extern "C" mote_status_t mote_moe_forward(const mote_layer_t* L, const void* x, 
       !L->alpha_up || !L->alpha_down || !L->sh_gate || !L->sh_up || !L->sh_down)
     return MOTE_ERR_NULL;
   if (x == out) return MOTE_ERR_SHAPE;
+  const int sh_bits = L->shared_bits == 0 ? MOTE_SHARED_BF16 : L->shared_bits;
+  if (sh_bits != MOTE_SHARED_BF16 && sh_bits != MOTE_SHARED_INT8 && sh_bits != MOTE_SHARED_INT4) return MOTE_ERR_SHAPE;
+  const bool sh_rtn = sh_bits != MOTE_SHARED_BF16;
+  if (sh_rtn && (!L->sh_gate_scale || !L->sh_up_scale || !L->sh_down_scale)) return MOTE_ERR_NULL;
+  const SharedMat sh_gate{L->sh_gate, sh_rtn ? L->sh_gate_scale : nullptr};
+  const SharedMat sh_up{L->sh_up, sh_rtn ? L->sh_up_scale : nullptr};
+  const SharedMat sh_down{L->sh_down, sh_rtn ? L->sh_down_scale : nullptr};
   const void* ptrs[] = {x, out, residual, L->Wr, L->gate_packed, L->up_packed, L->down_packed,
-                        L->sh_gate, L->sh_up, L->sh_down};
+                        L->sh_gate, L->sh_up, L->sh_down, sh_gate.scale, sh_up.scale, sh_down.scale};
   for (const void* p : ptrs)
     if (p && !aligned16(p)) return MOTE_ERR_ALIGN;
   if ((reinterpret_cast<uintptr_t>(ws) & 255u) != 0) return MOTE_ERR_ALIGN;
@@ -203,7 +210,7 @@ extern "C" mote_status_t mote_moe_forward(const mote_layer_t* L, const void* x, 
     ds.Wr = L->Wr; ds.router_bias = L->router_bias;
     ds.gate_packed = L->gate_packed; ds.up_packed = L->up_packed; ds.down_packed = L->down_packed;
     ds.alpha_gate = L->alpha_gate; ds.alpha_up = L->alpha_up; ds.alpha_down = L->alpha_down;
-    ds.sh_gate = L->sh_gate; ds.sh_up = L->sh_up; ds.sh_down = L->sh_down;
+    ds.sh_gate = sh_gate; ds.sh_up = sh_up; ds.sh_down = sh_down; ds.shared_bits = sh_bits;
     ds.topk_idx = topk_idx; ds.topk_w = topk_w; ds.offsets = offsets; ds.perm = perm; ds.inv = inv;
     ds.qx = qx; ds.beta_x = beta_x; ds.rowsum_x = rowsum_x; ds.h = h; ds.qh = qh; ds.beta_h = beta_h;
     ds.rowsum_h = rowsum_h; ds.y = y; ds.hs = hs; ds.s = s; ds.counter = status + 1;
@@ -307,21 +314,22 @@ extern "C" mote_status_t mote_moe_forward(const mote_layer_t* L, const void* x, 
   if (st) return st;
   stage_mark(6, stream);
   // S7 shared expert
-  st = tensor ? launch_shared_umma(x, L->sh_gate, L->sh_up, true, T, d, f, hs, tiles_shared, max_mtiles_shared,
+  st = tensor ? launch_shared_umma(x, sh_gate, sh_up, sh_bits, true, T, d, f, hs, tiles_shared, max_mtiles_shared,
                                    status, nullptr, stream, pdl)
-              : launch_shared_gateup_simt(x, L->sh_gate, L->sh_up, T, d, f, hs, stream);
+              : launch_shared_gateup_simt(x, sh_gate, sh_up, sh_bits, T, d, f, hs, stream);
   if (st) return st;
   stage_mark(7, stream);
   if (tensor) {
     // shared down projection with S8 (combine, residual, bf16 rounding) in its epilogue; the fp32
     // shared output is written only when a tap asks for it
     CombineArgs cb{y, topk_w, perm, residual, out, k};
-    st = launch_shared_umma(hs, L->sh_down, nullptr, false, T, f, d, (taps && taps->shared_out) ? s : nullptr,
-                            tiles_shared, max_mtiles_shared, status, &cb, stream, pdl);
+    st = launch_shared_umma(hs, sh_down, SharedMat{nullptr, nullptr}, sh_bits, false, T, f, d,
+                            (taps && taps->shared_out) ? s : nullptr, tiles_shared, max_mtiles_shared, status, &cb,
+                            stream, pdl);
     if (st) return st;
     stage_mark(8, stream);
   } else {
-    st = launch_shared_down_simt(hs, L->sh_down, T, d, f, s, stream);
+    st = launch_shared_down_simt(hs, sh_down, sh_bits, T, d, f, s, stream);
     if (st) return st;
     stage_mark(8, stream);
     // S8 combine

@@ -19,6 +19,30 @@
 
 namespace mote {
 
+// ------------------------------------------------------------------------------------------------
+// RTN codes of the shared expert (Section 4.3) -> bf16 operands of the tensor-core MMAs, exactly.
+// 0x4300 | m is the bf16 number 128 + m for a 7-bit m, so a code becomes a bf16 bit pattern with
+// byte moves and one exact bf16 subtraction.
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t sub_bf16x2(uint32_t a, uint32_t b) {
+  uint32_t d;
+  asm("sub.rn.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+  return d;
+}
+// four int8 codes (one word, memory order) -> bf16x2 of elements (0, 1) and (2, 3):
+// q = (q & 127) - 128 * signbit = (128 + (q & 127)) - (128 + 128 * signbit)
+__device__ __forceinline__ void s8x4_to_bf16x2(uint32_t w, uint32_t& e01, uint32_t& e23) {
+  const uint32_t m = w & 0x7F7F7F7Fu, sg = w & 0x80808080u;
+  e01 = sub_bf16x2(__byte_perm(m, 0x43434343u, 0x4140), __byte_perm(sg, 0x43434343u, 0x4140));
+  e23 = sub_bf16x2(__byte_perm(m, 0x43434343u, 0x4342), __byte_perm(sg, 0x43434343u, 0x4342));
+}
+// eight 4-bit codes (one word: nibble p = element 2p, nibble 4+p = element 2p+1, stored q + 8)
+// -> bf16x2 of elements (2p, 2p+1), p = 0..3:  q = (128 + u) - 136
+__device__ __forceinline__ void u4x8_to_bf16x2(uint32_t w, uint32_t (&e)[4]) {
+#pragma unroll
+  for (int p = 0; p < 4; ++p) e[p] = sub_bf16x2(((w >> (4 * p)) & 0x000F000Fu) | 0x43004300u, 0x43084308u);
+}
+
 // ---------------------------------------------------------------------------------------------
 // Programmatic dependent launch: a kernel launched with launch_pdl may start while the kernel
 // before it on the stream is still running; it calls pdl_wait() before it touches anything that

@@ -81,19 +81,24 @@ mote_status_t launch_ternary_umma(const TernaryGemmArgs& a, bool gateup, const i
 mote_status_t launch_quant_rows_known_beta(const void* h_bf16, int64_t rows, int n, int8_t* q, float* beta,
                                            int32_t* rowsum, int interleave, cudaStream_t stream, bool pdl = false,
                                            bool early_trigger = false);
+// One matrix of the shared expert: bf16 values (bits = 16, scale unused) or the codes of
+// mote_rtn_quant (bits = 8 or 4: int8 rows, or 4-bit codes in the pair-split word order) with one
+// scale per row.
+struct SharedMat { const void* w; const float* scale; };
+
 // comb (down projection only, may be null): fold the combine of Eq. 2 / Eq. 4 into the epilogue and
 // write the layer output directly; `out` (fp32 s) may then be null.
 struct CombineArgs {
   const float* y; const float* w; const int32_t* perm; const void* residual; void* out; int k;
 };
-mote_status_t launch_shared_umma(const void* act, const void* w0, const void* w1, bool gateup, int64_t T, int K,
-                                 int N, void* out, const int4* tiles, int max_mtiles, uint32_t* status,
-                                 const CombineArgs* comb, cudaStream_t stream, bool pdl = false);
+mote_status_t launch_shared_umma(const void* act, const SharedMat& w0, const SharedMat& w1, int bits, bool gateup,
+                                 int64_t T, int K, int N, void* out, const int4* tiles, int max_mtiles,
+                                 uint32_t* status, const CombineArgs* comb, cudaStream_t stream, bool pdl = false);
 
-// CUDA-core bf16 GEMMs of the shared expert.
-mote_status_t launch_shared_gateup_simt(const void* x, const void* Wg, const void* Wu, int64_t T, int d,
-                                        int f, void* h_bf16, cudaStream_t stream);
-mote_status_t launch_shared_down_simt(const void* h, const void* Wd, int64_t T, int d, int f, float* s,
+// CUDA-core GEMMs of the shared expert.
+mote_status_t launch_shared_gateup_simt(const void* x, const SharedMat& Wg, const SharedMat& Wu, int bits, int64_t T,
+                                        int d, int f, void* h_bf16, cudaStream_t stream);
+mote_status_t launch_shared_down_simt(const void* h, const SharedMat& Wd, int bits, int64_t T, int d, int f, float* s,
                                       cudaStream_t stream);
 
 // Decode path (T <= 64): prologue (Q_a(x), router, dispatch), streamed gate/up, Q_a(h), streamed
@@ -104,7 +109,7 @@ struct DecodeStreamArgs {
   const float* Wr; const float* router_bias;
   const uint8_t* gate_packed; const uint8_t* up_packed; const uint8_t* down_packed;
   const float* alpha_gate; const float* alpha_up; const float* alpha_down;
-  const void* sh_gate; const void* sh_up; const void* sh_down;
+  SharedMat sh_gate, sh_up, sh_down; int shared_bits;      // 16, 8 or 4
   int32_t* topk_idx; float* topk_w; int32_t* offsets; int32_t* perm; int32_t* inv;
   int8_t* qx; float* beta_x; int32_t* rowsum_x;
   void* h; int8_t* qh; float* beta_h; int32_t* rowsum_h; float* y; void* hs; float* s;

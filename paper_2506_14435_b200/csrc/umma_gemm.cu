@@ -6,6 +6,10 @@
 //   T_DOWN    routed down (Eq. 5): int8 Q_a(h) x 2-bit weights -> int32 -> y fp32
 //   B_GATEUP  shared expert gate/up (Eq. 2): bf16 x bf16 -> fp32 -> h_shared bf16
 //   B_DOWN    shared expert down -> s fp32
+//   Q8_*, Q4_* the same two with RTN INT8 / INT4 weight codes (Section 4.3): the codes travel to
+//             shared memory as stored, the unpacker warps expand them to bf16 (exact: |q| <= 127)
+//             in the swizzled operand layout, the MMA is the bf16 one and the epilogue multiplies
+//             every output column by its row scale
 //
 // Tile: 128 token rows (UMMA M, one TMEM lane per row) x BN weight rows (UMMA N = 256; for a down
 // projection the largest multiple of 32 up to 256 that divides its width, e.g. 224 for 896); K advances 128 bytes of the token
@@ -39,13 +43,13 @@ namespace mote {
 
 using namespace ptx;
 
-enum { MODE_T_GATEUP = 0, MODE_T_DOWN = 1, MODE_B_GATEUP = 2, MODE_B_DOWN = 3 };
+enum { MODE_T_GATEUP = 0, MODE_T_DOWN = 1, MODE_B_GATEUP = 2, MODE_B_DOWN = 3,
+       MODE_Q8_GATEUP = 4, MODE_Q8_DOWN = 5, MODE_Q4_GATEUP = 6, MODE_Q4_DOWN = 7 };
 
 constexpr int kBM = 128;
 constexpr int kStageA = kBM * 128;             // 16 KB: 128 rows x 128 B
 constexpr int kStageB = 256 * 128;             // 32 KB: up to 256 rows x 128 B
-constexpr int kStageP = 256 * 32;              // 8 KB: up to 256 rows x 32 B of packed codes
-constexpr int kStagesTernary = 3, kStagesP = 4, kStagesBf16 = 4;
+constexpr int kStagesTernary = 3, kStagesBf16 = 4, kStagesRtn = 3;
 constexpr int kThreads = 640;
 constexpr int kTmemCols = 512;
 
@@ -58,8 +62,8 @@ struct UmmaArgs {
   int b_rows_per_expert;    // rows of the weight tensor map per expert (0: shared expert)
   const float* beta;        // [rows]   (ternary modes)
   const int32_t* rowsum;    // [rows]
-  const float* alpha0;      // [E]
-  const float* alpha1;      // [E] (gate/up: alpha_up)
+  const float* alpha0;      // [E]; RTN modes: [n_out] scale of every output column
+  const float* alpha1;      // [E] (gate/up: alpha_up); RTN gate/up: [n_out] scales of the up matrix
   void* out;                // bf16 [rows, n_out] (gate/up) or fp32 [rows, n_out] (down)
   int32_t* tap0;            // optional int32 [rows, n_out]
   int32_t* tap1;
@@ -80,8 +84,15 @@ struct __align__(8) PipeBarriers {
 template <int MODE>
 struct ModeTraits {
   static constexpr bool kTernary = (MODE == MODE_T_GATEUP || MODE == MODE_T_DOWN);
-  static constexpr bool kGateUp = (MODE == MODE_T_GATEUP || MODE == MODE_B_GATEUP);
-  static constexpr int kStages = kTernary ? kStagesTernary : kStagesBf16;
+  static constexpr int kRtnBits = MODE >= MODE_Q4_GATEUP ? 4 : MODE >= MODE_Q8_GATEUP ? 8 : 0;
+  static constexpr bool kRtn = kRtnBits != 0;
+  static constexpr bool kUnpack = kTernary || kRtn;       // weights reach shared memory as codes
+  static constexpr bool kGateUp = (MODE % 2 == 0);
+  static constexpr int kStages = kTernary ? kStagesTernary : kRtn ? kStagesRtn : kStagesBf16;
+  // code bytes per weight row and pipeline stage: 128 2-bit codes, 64 int8 codes or 64 4-bit codes
+  static constexpr int kCodeRowBytes = kRtnBits == 8 ? 64 : 32;
+  static constexpr int kStageP = 256 * kCodeRowBytes;     // up to 256 rows
+  static constexpr int kStagesP = kRtnBits == 8 ? 3 : 4;
   // gate/up epilogue: every epilogue warp stages 32 rows x kEpiCols bf16 (row pitch padded by 16 B)
   // and writes them out as whole row segments
   // (bf16 gate/up only.  For the ternary gate/up, whose epilogue competes with the unpackers for
@@ -91,7 +102,7 @@ struct ModeTraits {
   static constexpr int kEpiPitch = kEpiCols * 2 + 16;
   static constexpr size_t kEpiStage = (kGateUp && !kTernary) ? size_t(8) * 32 * kEpiPitch : 0;
   static constexpr size_t kSmem = 1024 + size_t(kStages) * (kStageA + kStageB) +
-                                  (kTernary ? size_t(kStagesP) * kStageP : 0) + kEpiStage + sizeof(PipeBarriers);
+                                  (kUnpack ? size_t(kStagesP) * kStageP : 0) + kEpiStage + sizeof(PipeBarriers);
 };
 
 // Item order.  The CTAs of the grid work on neighbouring items at the same time, and the operand
@@ -123,7 +134,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
   const uint32_t sP = sB + S * kStageB;
   uint8_t* genB = smem_gen + S * kStageA;
   uint8_t* genP = genB + S * kStageB;
-  uint8_t* genE = genP + (TR::kTernary ? kStagesP * kStageP : 0);
+  uint8_t* genE = genP + (TR::kUnpack ? TR::kStagesP * TR::kStageP : 0);
   PipeBarriers* bars = reinterpret_cast<PipeBarriers*>(genE + TR::kEpiStage);
   volatile int* abort_flag = &bars->abort_flag;
 
@@ -174,6 +185,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
           if (TR::kTernary) {
             mbar_expect_tx(bar, kStageA);
             tma_load_2d(sA + stage * kStageA, &tm_a, ks * 128, tile.y, bar);
+          } else if (TR::kRtn) {
+            mbar_expect_tx(bar, kStageA);
+            tma_load_2d(sA + stage * kStageA, &tm_a, ks * 64, tile.y, bar);
           } else {
             mbar_expect_tx(bar, kStageA + a.bn * 128);
             tma_load_2d(sA + stage * kStageA, &tm_a, ks * 64, tile.y, bar);
@@ -191,7 +205,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
     }
   } else if (warp == 1) {
     // ---------------------------------------------------------------- packed-weight producer
-    if (TR::kTernary && lane == 0) {
+    if (TR::kUnpack && lane == 0) {
+      constexpr int kRB = TR::kCodeRowBytes;
       uint32_t stage = 0, phase = 0;
       bool ok = true;
       for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x) {
@@ -201,16 +216,16 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
         for (int ks = 0; ks < a.k_steps; ++ks) {
           if (!(ok = mbar_wait(smem_u32(&bars->empty_p[stage]), phase ^ 1, abort_flag))) break;
           const uint32_t bar = smem_u32(&bars->full_p[stage]);
-          mbar_expect_tx(bar, a.bn * 32);
-          const uint32_t dst = sP + stage * kStageP;
+          mbar_expect_tx(bar, a.bn * kRB);
+          const uint32_t dst = sP + stage * TR::kStageP;
           if (TR::kGateUp) {
-            tma_load_2d(dst, &tm_b0, ks * 32, b_row, bar);
-            tma_load_2d(dst + 128 * 32, &tm_b1, ks * 32, b_row, bar);
+            tma_load_2d(dst, &tm_b0, ks * kRB, b_row, bar);
+            tma_load_2d(dst + 128 * kRB, &tm_b1, ks * kRB, b_row, bar);
           } else {
-            tma_load_2d(dst, &tm_b0, ks * 32, b_row, bar);
-            if (a.bn > 128) tma_load_2d(dst + 128 * 32, &tm_b1, ks * 32, b_row + 128, bar);
+            tma_load_2d(dst, &tm_b0, ks * kRB, b_row, bar);
+            if (a.bn > 128) tma_load_2d(dst + 128 * kRB, &tm_b1, ks * kRB, b_row + 128, bar);
           }
-          if (++stage == kStagesP) { stage = 0; phase ^= 1; }
+          if (++stage == TR::kStagesP) { stage = 0; phase ^= 1; }
         }
       }
     }
@@ -230,7 +245,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
         const uint32_t d_tmem = tmem_base + buf * 256;
         for (int ks = 0; ks < a.k_steps; ++ks) {
           if (!(ok = mbar_wait(smem_u32(&bars->full_a[stage]), phase, abort_flag))) break;
-          if (TR::kTernary)
+          if (TR::kUnpack)
             if (!(ok = mbar_wait(smem_u32(&bars->full_u[stage]), phase, abort_flag))) break;
           tc_fence_after();
           const uint64_t da = smem_desc_sw128(sA + stage * kStageA);
@@ -248,14 +263,15 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
       }
     }
   } else if (warp >= 4 && warp < 12) {
-    // ---------------------------------------------------------------- 2-bit -> int8 unpackers
+    // ---------------------------------------------------------------- code unpackers
+    // (2-bit -> int8 for the ternary experts; int8 / 4-bit -> bf16 for an RTN-coded shared expert)
     // group 0 (warps 4-7) expands the even pipeline steps, group 1 (warps 8-11) the odd ones
-    if (TR::kTernary) {
+    if (TR::kUnpack) {
       const int group = (warp - 4) >> 2;
       const int tid = (threadIdx.x - 128) & 127;
       uint32_t stage = 0, phase = 0, pstage = 0, pphase = 0, step = 0;
       bool ok = true;
-      const int n_chunks = a.bn * 2;                 // chunks of 16 packed bytes, spread over 128 threads
+      const int n_chunks = a.bn * (TR::kCodeRowBytes / 16);   // chunks of 16 code bytes, spread over 128 threads
       for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x) {
         for (int ks = 0; ks < a.k_steps; ++ks, ++step) {
           if ((step & 1u) == (uint32_t)group) {
@@ -263,21 +279,39 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
                  mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1, abort_flag);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
-            const uint8_t* src = genP + pstage * kStageP;
+            const uint8_t* src = genP + pstage * TR::kStageP;
             uint8_t* dst = genB + stage * kStageB;
             for (int c = tid; c < n_chunks; c += 128) {
-              const int r = c >> 1, half = c & 1;
               const uint4 w = *reinterpret_cast<const uint4*>(src + c * 16);
               const uint32_t pw[4] = {w.x, w.y, w.z, w.w};
-              uint8_t* row = dst + (r >> 3) * 1024 + (r & 7) * 128;
+              if (TR::kRtnBits == 8) {
+                // 16 int8 codes -> two 16-byte pieces of 8 bf16 each
+                const int r = c >> 2, quarter = c & 3;
+                uint8_t* row = dst + (r >> 3) * 1024 + (r & 7) * 128;
+                uint32_t e[8];
 #pragma unroll
-              for (int j = 0; j < 4; ++j) {
-                uint4 o;
-                o.x = pw[j] & 0x03030303u;
-                o.y = (pw[j] >> 2) & 0x03030303u;
-                o.z = (pw[j] >> 4) & 0x03030303u;
-                o.w = (pw[j] >> 6) & 0x03030303u;
-                *reinterpret_cast<uint4*>(row + (((half * 4 + j) ^ (r & 7)) << 4)) = o;
+                for (int j = 0; j < 4; ++j) s8x4_to_bf16x2(pw[j], e[2 * j], e[2 * j + 1]);
+                *reinterpret_cast<uint4*>(row + (((quarter * 2) ^ (r & 7)) << 4)) = make_uint4(e[0], e[1], e[2], e[3]);
+                *reinterpret_cast<uint4*>(row + (((quarter * 2 + 1) ^ (r & 7)) << 4)) = make_uint4(e[4], e[5], e[6], e[7]);
+              } else {
+                const int r = c >> 1, half = c & 1;
+                uint8_t* row = dst + (r >> 3) * 1024 + (r & 7) * 128;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                  uint4 o;
+                  if (TR::kRtnBits == 4) {
+                    // 8 four-bit codes -> one 16-byte piece of 8 bf16
+                    uint32_t e[4];
+                    u4x8_to_bf16x2(pw[j], e);
+                    o = make_uint4(e[0], e[1], e[2], e[3]);
+                  } else {
+                    o.x = pw[j] & 0x03030303u;
+                    o.y = (pw[j] >> 2) & 0x03030303u;
+                    o.z = (pw[j] >> 4) & 0x03030303u;
+                    o.w = (pw[j] >> 6) & 0x03030303u;
+                  }
+                  *reinterpret_cast<uint4*>(row + (((half * 4 + j) ^ (r & 7)) << 4)) = o;
+                }
               }
             }
             fence_proxy_async_smem();                // generic-proxy writes -> visible to the MMA
@@ -288,7 +322,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
             }
           }
           if (++stage == S) { stage = 0; phase ^= 1; }
-          if (++pstage == kStagesP) { pstage = 0; pphase ^= 1; }
+          if (++pstage == TR::kStagesP) { pstage = 0; pphase ^= 1; }
         }
       }
     }
@@ -352,6 +386,20 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
                 }
 #pragma unroll
                 for (int j = 0; j < 16; ++j) hmax = fmaxf(hmax, fabsf(hv[j]));
+              } else if (TR::kRtn) {
+                // row scales of the gate and up matrices = scales of this tile's output columns
+                const float4* sgp = reinterpret_cast<const float4*>(a.alpha0 + col0 + c);
+                const float4* sup = reinterpret_cast<const float4*>(a.alpha1 + col0 + c);
+#pragma unroll
+                for (int v = 0; v < 4; ++v) {
+                  const float4 sg = __ldg(sgp + v), su = __ldg(sup + v);
+                  const float sgv[4] = {sg.x, sg.y, sg.z, sg.w}, suv[4] = {su.x, su.y, su.z, su.w};
+#pragma unroll
+                  for (int u = 0; u < 4; ++u) {
+                    const float g = __uint_as_float(rg[4 * v + u]) * sgv[u];
+                    hv[4 * v + u] = __uint_as_float(ru[4 * v + u]) * suv[u] * silu_fast(g);
+                  }
+                }
               } else {
 #pragma unroll
                 for (int j = 0; j < 16; ++j) {
@@ -426,6 +474,14 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
 #pragma unroll
             for (int v = 0; v < 16; ++v)
               o[v] = TR::kTernary ? __fmul_rn(i2f_small((int)ra[v] - rs), c0) : __uint_as_float(ra[v]);
+            if (TR::kRtn) {
+              const float4* sp = reinterpret_cast<const float4*>(a.alpha0 + col0 + c);
+#pragma unroll
+              for (int v = 0; v < 4; ++v) {
+                const float4 sc = __ldg(sp + v);
+                o[4 * v] *= sc.x; o[4 * v + 1] *= sc.y; o[4 * v + 2] *= sc.z; o[4 * v + 3] *= sc.w;
+              }
+            }
             if (a.out) {
               float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(a.out) + row * a.n_out + col0 + c);
 #pragma unroll
@@ -586,21 +642,33 @@ mote_status_t launch_ternary_umma(const TernaryGemmArgs& g, bool gateup, const i
                 : launch_umma<MODE_T_DOWN>(ta, tb0, tb1, a, max_items, stream, pdl);
 }
 
-mote_status_t launch_shared_umma(const void* act, const void* w0, const void* w1, bool gateup, int64_t T, int K,
-                                 int N, void* out, const int4* tiles, int max_mtiles, uint32_t* status,
-                                 const CombineArgs* comb, cudaStream_t stream, bool pdl) {
+mote_status_t launch_shared_umma(const void* act, const SharedMat& w0, const SharedMat& w1, int bits, bool gateup,
+                                 int64_t T, int K, int N, void* out, const int4* tiles, int max_mtiles,
+                                 uint32_t* status, const CombineArgs* comb, cudaStream_t stream, bool pdl) {
   if (T == 0) return MOTE_OK;
   CUtensorMap ta, tb0, tb1;
   const int bn = gateup ? 256 : pick_bn(N);
+  const uint32_t rows1 = (gateup || bn <= 128) ? 128 : bn - 128;
   if (!make_map_2d(&ta, act, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)T, (uint64_t)K, 128, 64,
                    CU_TENSOR_MAP_SWIZZLE_128B))
     return MOTE_ERR_CUDA;
-  if (!make_map_2d(&tb0, w0, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)N, (uint64_t)K, 128, 64,
-                   CU_TENSOR_MAP_SWIZZLE_128B))
-    return MOTE_ERR_CUDA;
-  if (!make_map_2d(&tb1, gateup ? w1 : w0, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)N, (uint64_t)K,
-                   (gateup || bn <= 128) ? 128 : bn - 128, 64, CU_TENSOR_MAP_SWIZZLE_128B))
-    return MOTE_ERR_CUDA;
+  const void* wb1 = gateup ? w1.w : w0.w;
+  if (bits == 16) {
+    if (!make_map_2d(&tb0, w0.w, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)N, (uint64_t)K, 128, 64,
+                     CU_TENSOR_MAP_SWIZZLE_128B) ||
+        !make_map_2d(&tb1, wb1, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (uint64_t)N, (uint64_t)K, rows1, 64,
+                     CU_TENSOR_MAP_SWIZZLE_128B))
+      return MOTE_ERR_CUDA;
+  } else {
+    // code rows as bytes: K (int8) or K/2 (4-bit) per row, 64 reduction elements per pipeline stage
+    const uint64_t row_bytes = bits == 8 ? (uint64_t)K : (uint64_t)K / 2;
+    const uint32_t box = bits == 8 ? 64 : 32;
+    if (!make_map_2d(&tb0, w0.w, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)N, row_bytes, 128, box,
+                     CU_TENSOR_MAP_SWIZZLE_NONE) ||
+        !make_map_2d(&tb1, wb1, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)N, row_bytes, rows1, box,
+                     CU_TENSOR_MAP_SWIZZLE_NONE))
+      return MOTE_ERR_CUDA;
+  }
   UmmaArgs a{};
   a.tiles = tiles;
   a.n_ntiles = gateup ? N / 128 : N / bn;
@@ -610,12 +678,19 @@ mote_status_t launch_shared_umma(const void* act, const void* w0, const void* w1
   a.b_rows_per_expert = 0;
   a.out = out;
   a.status = status;
+  a.alpha0 = w0.scale; a.alpha1 = w1.scale;     // RTN modes only
   if (comb && !gateup) {
     a.comb_y = comb->y; a.comb_w = comb->w; a.comb_perm = comb->perm;
     a.comb_res = static_cast<const uint16_t*>(comb->residual); a.comb_out = static_cast<uint16_t*>(comb->out);
     a.comb_k = comb->k;
   }
   const int max_items = max_mtiles * a.n_ntiles;
+  if (bits == 8)
+    return gateup ? launch_umma<MODE_Q8_GATEUP>(ta, tb0, tb1, a, max_items, stream, pdl)
+                  : launch_umma<MODE_Q8_DOWN>(ta, tb0, tb1, a, max_items, stream, pdl);
+  if (bits == 4)
+    return gateup ? launch_umma<MODE_Q4_GATEUP>(ta, tb0, tb1, a, max_items, stream, pdl)
+                  : launch_umma<MODE_Q4_DOWN>(ta, tb0, tb1, a, max_items, stream, pdl);
   return gateup ? launch_umma<MODE_B_GATEUP>(ta, tb0, tb1, a, max_items, stream, pdl)
                 : launch_umma<MODE_B_DOWN>(ta, tb0, tb1, a, max_items, stream, pdl);
 }

@@ -82,3 +82,15 @@ def check_forward(mote, layer_gpu, layer_or: dict, x_bits: np.ndarray, residual_
     assert err <= REL_FRO_TOL, err
     return dict(rel_fro=err, shared_rel_fro=sh_err, near_ties=int(near.sum()), tokens=len(toks),
                 out=out, counts=np.diff(ref["offsets"]))
+
+
+def check_shared_codes(layer_gpu, layer_or: dict):
+    """RTN codes and row scales of the shared expert (Section 4.3): bit-exact."""
+    rtn = layer_or["sh_rtn"]
+    assert layer_gpu.shared_bits == rtn["bits"]
+    for name in ("gate", "up", "down"):
+        q, scale = rtn[name]
+        got = layer_gpu.tensors["sh_" + name].cpu().numpy()
+        want = q if rtn["bits"] == 8 else O.pack_int4(q)
+        assert got.dtype == want.dtype and np.array_equal(got, want), name
+        assert np.array_equal(layer_gpu.tensors["sh_" + name + "_scale"].cpu().numpy(), scale), name

@@ -76,10 +76,23 @@ def test_host_side_argument_errors(mote):
     assert lib.mote_moe_forward(C.byref(L), NULL, NULL, 0, NULL, None, NULL, 0, NULL) == 0       # T = 0
     Lbad = mote_layer_t(250, 512, 4, 2, 1, 0)
     assert lib.mote_moe_forward(C.byref(Lbad), fake, NULL, 4, fake, None, ws, 1 << 30, NULL) == 2
-    for name, _ in mote_layer_t._fields_[6:]:
-        setattr(L, name, 0x2000)
+    for name, ctype in mote_layer_t._fields_[6:]:
+        if ctype is C.c_void_p:
+            setattr(L, name, 0x2000)
     L.router_bias = None
     assert lib.mote_moe_forward(C.byref(L), fake, NULL, 4, fake, None, ws, 1 << 30, NULL) == 2   # out aliases x
     other = C.c_void_p(0x3000)
     assert lib.mote_moe_forward(C.byref(L), fake, NULL, 4, other, None, ws, 16, NULL) == 4       # workspace
     assert lib.mote_moe_forward(C.byref(L), fake, NULL, 4, other, None, C.c_void_p(0x10010), 1 << 30, NULL) == 3
+    # shared-expert storage: unknown width, RTN codes without their scales
+    L.shared_bits = 5
+    assert lib.mote_moe_forward(C.byref(L), fake, NULL, 4, other, None, ws, 1 << 30, NULL) == 2
+    L.shared_bits = 4
+    L.sh_down_scale = None
+    assert lib.mote_moe_forward(C.byref(L), fake, NULL, 4, other, None, ws, 1 << 30, NULL) == 1
+    # rtn_quant
+    assert lib.mote_rtn_quant(NULL, 1, 4, 16, 8, fake, fake, NULL) == 1
+    assert lib.mote_rtn_quant(fake, 9, 4, 16, 8, fake, fake, NULL) == 5
+    assert lib.mote_rtn_quant(fake, 1, 4, 24, 8, fake, fake, NULL) == 2
+    assert lib.mote_rtn_quant(fake, 1, 4, 16, 2, fake, fake, NULL) == 2
+    assert lib.mote_rtn_quant(odd, 1, 4, 16, 4, fake, fake, NULL) == 3

@@ -6,7 +6,7 @@ import torch
 
 from oracle import mote_oracle as O
 from workloads import synth
-from parity_utils import bf16_bits, bf16_tensor, check_forward, check_packed_layer
+from parity_utils import bf16_bits, bf16_tensor, check_forward, check_packed_layer, check_shared_codes
 
 pytestmark = pytest.mark.gpu
 
@@ -154,3 +154,53 @@ def test_host_buffer_entry_point(mote):
     mote_moe_forward_host(layer_gpu, x_host, out_host)
     want = mote.mote_moe_forward(layer_gpu, x_host.cuda())
     assert torch.equal(out_host, want.cpu())
+
+
+# ------------------------------------------------------------------ Section 4.3: RTN-coded shared expert
+@pytest.mark.parametrize("bits", [8, 4])
+@pytest.mark.parametrize("d,f,E,k,T,kw,path", [
+    (16, 32, 3, 2, 5, {}, SIMT),
+    (64, 112, 5, 5, 33, {}, SIMT),
+    (128, 128, 2, 1, 1, {}, TENSOR),                      # one row, two k-steps
+    (256, 512, 4, 2, 300, dict(outlier_frac=0.02), TENSOR),
+    (128, 384, 4, 1, 130, dict(norm_topk=0), TENSOR),     # down projection with 128-wide tiles
+    (384, 640, 3, 3, 515, {}, TENSOR),                    # several row tiles, 160-wide down tiles (128 + 32 rows)
+    (896, 4864, 4, 2, 160, dict(outlier_frac=0.01), TENSOR),  # 224-wide down tiles
+    (64, 128, 3, 3, 5, {}, STREAM),                       # one short reduction step (32 bytes of 4-bit codes)
+    (128, 192, 2, 1, 1, {}, STREAM),
+    (896, 4864, 4, 2, 17, dict(outlier_frac=0.01), STREAM),
+    (256, 512, 4, 2, 64, dict(bias="zipf"), STREAM),
+])
+def test_rtn_shared_expert(mote, d, f, E, k, T, kw, path, bits):
+    wl = synth.custom("rtn", d, f, E, k, T, 4000 + d + f + T, **kw)
+    master, layer_or, layer_gpu = _setup(mote, wl, path)
+    layer_or = O.quantize_shared(layer_or, bits)
+    layer_gpu = layer_gpu.quantize_shared(bits)
+    check_shared_codes(layer_gpu, layer_or)
+    check_forward(mote, layer_gpu, layer_or, synth.tokens(wl))
+
+
+@pytest.mark.parametrize("bits", [8, 4])
+@pytest.mark.parametrize("path", ALL)
+def test_rtn_shared_expert_c3_decode(mote, path, bits, c3_layers):
+    wl, layer_or, layer_gpu = c3_layers
+    layer_or = O.quantize_shared(layer_or, bits)
+    layer_q = layer_gpu.quantize_shared(bits, path=path)
+    check_shared_codes(layer_q, layer_or)
+    for T in (1, 33):
+        rep = check_forward(mote, layer_q, layer_or, synth.tokens(wl, T=T))
+        assert rep["rel_fro"] < 5e-3
+
+
+def test_rtn_shared_expert_rejects_missing_scales(mote):
+    wl = synth.WORKLOADS["c1"]
+    master, layer_or, layer_gpu = _setup(mote, wl)
+    layer_q = layer_gpu.quantize_shared(8)
+    layer_q.tensors["sh_up_scale"] = None
+    with pytest.raises(mote.MoteError) as ei:
+        mote.mote_moe_forward(layer_q, bf16_tensor(synth.tokens(wl)))
+    assert ei.value.status == 1
+    layer_gpu.shared_bits = 5
+    with pytest.raises(mote.MoteError) as ei:
+        mote.mote_moe_forward(layer_gpu, bf16_tensor(synth.tokens(wl)))
+    assert ei.value.status == 2

@@ -139,3 +139,44 @@ def test_quant_act_every_bf16_value_under_many_scales(mote):
     assert np.array_equal(gb.cpu().numpy(), beta)
     assert np.array_equal(gq.cpu().numpy(), q)
     assert np.array_equal(gs.cpu().numpy(), rowsum)
+
+
+@pytest.mark.parametrize("bits", [8, 4])
+@pytest.mark.parametrize("m,n,scale,dtype", [(1, 16, 0.02, "bf16"), (7, 48, 0.02, "f32"), (300, 1008, 1.0, "bf16"),
+                                             (129, 11008, 0.02, "bf16"), (64, 896, 0.02, "f32"),
+                                             (33, 65536, 0.02, "bf16"), (16, 64, 1e-30, "f32")])
+def test_rtn_quant(mote, m, n, scale, dtype, bits):
+    W = _randn((m, n), 900 + m + n + bits, scale).astype(np.float32)
+    if m > 4:
+        W[3] = 0.0                                  # an all-zero row
+    if dtype == "bf16":
+        Wb = O.f32_to_bf16_rn(W)
+        q_ref, s_ref = O.rtn_quantize(O.bf16_to_f32(Wb), bits)
+        q, sc = mote.mote_rtn_quant(bf16_tensor(Wb), bits)
+    else:
+        q_ref, s_ref = O.rtn_quantize(W, bits)
+        q, sc = mote.mote_rtn_quant(torch.from_numpy(W).cuda(), bits)
+    want = q_ref if bits == 8 else O.pack_int4(q_ref)
+    assert np.array_equal(q.cpu().numpy(), want)
+    assert np.array_equal(sc.cpu().numpy(), s_ref)
+
+
+@pytest.mark.parametrize("bits", [8, 4])
+def test_rtn_quant_ties_and_errors(mote, bits):
+    # exact half-integer quotients: rows of k + 1/2 multiples of beta/qmax
+    qmax = 2 ** (bits - 1) - 1
+    base = np.arange(-qmax, qmax + 1, dtype=np.float32)
+    row = np.concatenate([base, base[:-1] + 0.5])
+    row = np.resize(row, 64).astype(np.float32)
+    row[0] = qmax
+    W = np.tile(row, (5, 1)) * np.float32(0.125)
+    q_ref, s_ref = O.rtn_quantize(W, bits)
+    q, sc = mote.mote_rtn_quant(torch.from_numpy(W).cuda(), bits)
+    assert np.array_equal(q.cpu().numpy(), q_ref if bits == 8 else O.pack_int4(q_ref))
+    assert np.array_equal(sc.cpu().numpy(), s_ref)
+    with pytest.raises(mote.MoteError) as ei:
+        mote.mote_rtn_quant(torch.zeros((4, 24), device="cuda"), bits)       # n % 16 != 0
+    assert ei.value.status == 2
+    with pytest.raises(mote.MoteError) as ei:
+        mote.mote_rtn_quant(torch.zeros((4, 32), device="cuda"), 3)
+    assert ei.value.status == 2
