@@ -2,6 +2,7 @@
 """Benchmark of the MoTE FFN-layer forward pass on B200.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2|c4|c3-T|c1] [--impl ours|reference]
+                  [--shared-bits 16|8|4]
 
 One "step" is one pass of the whole layer (route, dispatch, Q_a(x), gate/up ternary GEMM, Q_a(h),
 down ternary GEMM, shared bf16 FFN, combine) over one batch of synthetic tokens.  Weights are
@@ -99,21 +100,21 @@ class ClockSampler:
 
 # ncu dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the captures
 # summarised under profiles/ (null once the kernel has changed since, or where no capture exists)
-NCU_TRAFFIC_BYTES = {("c2", "gateup_ternary"): 43.31e6, ("c4", "gateup_ternary"): 584.32e6,
-                     ("c3-1", "gateup_ternary"): 70.70e6}
+NCU_TRAFFIC_BYTES = {}
 
 
-def stage_work(wl: synth.Workload, stage: str, stream_path: bool, experts_touched: float):
+def stage_work(wl: synth.Workload, stage: str, stream_path: bool, experts_touched: float, shared_bits: int = 16):
     """Algorithmic work of one launch of a stage: (amount, kind), kind 'int8' | 'bf16' | 'bytes'.
     On the decode path the gate/up and down stages each cover the routed AND the shared expert and
     are bound by the weight bytes they stream: 2-bit codes of the experts that received tokens plus
-    the bf16 shared matrices."""
+    the shared matrices (bf16, or RTN codes of shared_bits bits)."""
     P, T, d, f = wl.T * wl.k, wl.T, wl.d, wl.f
+    sh_bytes = shared_bits / 8.0
     if stream_path:
         if stage == "gateup_ternary":
-            return experts_touched * 2 * f * d / 4 + 2.0 * f * d * 2, "bytes"
+            return experts_touched * 2 * f * d / 4 + 2.0 * f * d * sh_bytes, "bytes"
         if stage == "down_ternary":
-            return experts_touched * f * d / 4 + f * d * 2.0, "bytes"
+            return experts_touched * f * d / 4 + f * d * sh_bytes, "bytes"
     if stage == "gateup_ternary":
         return 2.0 * P * d * 2 * f, "int8"
     if stage == "down_ternary":
@@ -181,6 +182,11 @@ def run_ours(args):
         x_bits = synth.tokens(wl, stream=rank)
         x_host = torch.from_numpy(x_bits.view(np.int16).copy()).view(torch.bfloat16).pin_memory()
         x = x_host.to(dev)
+    if args.shared_bits != 16:                          # offline step: RTN codes of the shared expert
+        layers = [l.quantize_shared(args.shared_bits) for l in layers]
+        if is_stack:
+            stack = mote.MoteStack(layers)
+        torch.cuda.empty_cache()
     out_host = torch.empty_like(x_host).pin_memory()
     out = torch.empty_like(x)
     flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
@@ -287,7 +293,7 @@ def run_ours(args):
     tokens_per_s = job_tokens_per_s(world, wl.T, args.steps, total_ms)
     decode = wl.T <= 64
     dom = max(stage_ms, key=stage_ms.get)
-    work, kind = stage_work(wl, dom, stream_path, experts_touched)
+    work, kind = stage_work(wl, dom, stream_path, experts_touched, args.shared_bits)
     dur_s = stage_ms[dom] * 1e-3 / len(layers)          # average duration of one launch of that kernel
     if kind == "bytes":
         roof = dict(bound="hbm", achieved=work / dur_s / 1e9, peak=peaks["hbm_gbs"], unit="GB/s")
@@ -301,7 +307,7 @@ def run_ours(args):
     roof["algorithmic_work_per_launch"] = work
     roof["peak_source"] = ("of measured" if peaks["source"] == "measured" else "of fallback") + \
         (" (bf16 burst x2 nominal int8:bf16 ratio)" if kind == "int8" else "")
-    weight_bytes = len(layers) * (experts_touched * 3 * wl.d * wl.f / 4 + 6.0 * wl.d * wl.f)
+    weight_bytes = len(layers) * (experts_touched * 3 * wl.d * wl.f / 4 + 3.0 * wl.d * wl.f * args.shared_bits / 8)
     if not bool(torch.isfinite(out.float()).all()):
         raise SystemExit("non-finite layer output: the timing would not be valid")
     line = {
@@ -309,9 +315,11 @@ def run_ours(args):
         "value": tokens_per_s, "unit": "tokens/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "us_per_layer": ms_per_step * 1e3 / len(layers),
         "us_per_token": ms_per_step * 1e3 / wl.T, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "int8xint2->int32 routed, bf16 shared", "data": "synthetic",
+        "scaling": "weak", "vs_baseline": None, "dtype": "int8xint2->int32 routed, bf16 shared" + (
+            "" if args.shared_bits == 16 else f" (weights RTN int{args.shared_bits}, weight-only)"), "data": "synthetic",
         "config": {"workload": wl.name, "d": wl.d, "f": wl.f, "E": wl.E, "k": wl.k, "T_per_gpu": wl.T,
                    "layers": len(layers), "experts_touched_per_layer": experts_touched,
+                   "shared_bits": args.shared_bits,
                    "pre_norm": "rms, eps 1e-6, unit gain" if is_stack else "none (the caller's)",
                    "l2": "flushed between timed iterations (512 MiB write)", "parallelism": f"replicas x{world}"},
         "stage_ms": stage_ms, "roofline": roof,
@@ -324,7 +332,7 @@ def run_ours(args):
         if is_stack:                                    # the oracle needs host-drawn weights: layer 0, scaled by the depth
             master = synth.master_layer(wl)
             x_bits = synth.tokens(wl)
-        cb = cpu_baseline(wl, master, x_bits, budget_s=12.0)
+        cb = cpu_baseline(wl, master, x_bits, budget_s=12.0, shared_bits=args.shared_bits)
         if is_stack:
             cb["value"] /= len(layers)
             cb["sample"] += f"; one layer timed, value divided by the {len(layers)} layers of the stack"
@@ -335,11 +343,13 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
-def cpu_baseline(wl, master, x_bits, budget_s: float, n_tokens: int | None = None):
+def cpu_baseline(wl, master, x_bits, budget_s: float, n_tokens: int | None = None, shared_bits: int = 16):
     """The oracle as it stands, on the host cores, on a bounded sample of the same workload: a
     short probe fixes the sample size so that the timed run takes about `budget_s` seconds."""
     from oracle import mote_oracle as O
     layer_or = O.build_layer(master)                     # offline step, not timed (as on the GPU)
+    if shared_bits != 16:
+        layer_or = O.quantize_shared(layer_or, shared_bits)
     n0 = min(wl.T, 32)
     t0 = time.perf_counter()
     O.moe_forward(layer_or, x_bits, token_subset=np.arange(n0))
@@ -362,6 +372,8 @@ def run_reference(args):
     master = synth.master_layer(wl)
     from oracle import mote_oracle as O
     layer_or = O.build_layer(master)
+    if args.shared_bits != 16:
+        layer_or = O.quantize_shared(layer_or, args.shared_bits)
     x_bits = synth.tokens(wl)
     n = min(wl.T, 128 if wl.d * wl.f < 8e6 else 32)
     sub = np.arange(n)
@@ -379,7 +391,8 @@ def run_reference(args):
         "value": val, "unit": "tokens/s", "n_gpus": int(os.environ.get("WORLD_SIZE", 1)), "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "fp64 / exact integers", "data": "synthetic",
-        "config": {"workload": wl.name, "d": wl.d, "f": wl.f, "E": wl.E, "k": wl.k, "T_per_gpu": wl.T},
+        "config": {"workload": wl.name, "d": wl.d, "f": wl.f, "E": wl.E, "k": wl.k, "T_per_gpu": wl.T,
+                   "shared_bits": args.shared_bits},
         "cpu_baseline": {"value": val, "unit": "tokens/s", "cores": torch.get_num_threads(), "kind": "oracle",
                          "sample": f"each step = first {n} of {wl.T} tokens of {wl.name}"},
         "e2e": {"value": val, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -393,6 +406,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="c2")
     ap.add_argument("--layers", type=int, default=None, help="layers of a stacked workload (c5-T: default 36)")
+    ap.add_argument("--shared-bits", type=int, default=16, choices=[16, 8, 4],
+                    help="storage of the shared expert: bf16, or RTN INT8 / INT4 codes (Section 4.3)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup

@@ -10,7 +10,7 @@ import torch
 
 from oracle import mote_oracle as O
 from workloads import synth
-from parity_utils import bf16_tensor, check_forward, check_packed_layer
+from parity_utils import bf16_tensor, check_forward, check_packed_layer, check_shared_codes
 
 pytestmark = pytest.mark.gpu
 
@@ -21,11 +21,15 @@ def mote():
     return m
 
 
-def _sampled_parity(mote, wl, n_random, max_boundary_tokens):
+def _sampled_parity(mote, wl, n_random, max_boundary_tokens, shared_bits=16):
     master = synth.master_layer(wl)
     layer_or = O.build_layer(master)
     layer_gpu = mote.MoteLayer.from_master(master)
     check_packed_layer(layer_gpu, layer_or)
+    if shared_bits != 16:
+        layer_or = O.quantize_shared(layer_or, shared_bits)
+        layer_gpu = layer_gpu.quantize_shared(shared_bits)
+        check_shared_codes(layer_gpu, layer_or)
     x_bits = synth.tokens(wl)
     r = O.router(x_bits, layer_or["Wr"], layer_or.get("router_bias"), wl.k, wl.norm_topk)
     offsets, perm, inv = O.dispatch(r["idx"], wl.E)
@@ -41,6 +45,12 @@ def _sampled_parity(mote, wl, n_random, max_boundary_tokens):
 
 def test_c2_full_size_sampled(mote):
     rep = _sampled_parity(mote, synth.WORKLOADS["c2"], n_random=96, max_boundary_tokens=400)
+    assert rep["rel_fro"] < 5e-3
+
+
+@pytest.mark.parametrize("bits", [8, 4])
+def test_c2_full_size_sampled_rtn_shared_expert(mote, bits):
+    rep = _sampled_parity(mote, synth.WORKLOADS["c2"], n_random=64, max_boundary_tokens=100, shared_bits=bits)
     assert rep["rel_fro"] < 5e-3
 
 
@@ -60,3 +70,16 @@ def test_paper_configuration_top1_full_softmax_gate(mote, T):
     rep = check_forward(mote, layer_gpu, layer_or, synth.tokens(wl))
     assert rep["rel_fro"] < 5e-3
     assert rep["counts"].sum() == T
+
+
+@pytest.mark.parametrize("bits", [8, 4])
+def test_paper_3b_layer_rtn_shared_expert_decode_and_prefill(mote, bits):
+    # the operating points of the paper's Table 3: the 3B model's layer with the shared expert in INT8 / INT4
+    wl = synth.WORKLOADS["p3"]
+    master = synth.master_layer(wl)
+    layer_or = O.quantize_shared(O.build_layer(master), bits)
+    layer_gpu = mote.MoteLayer.from_master(master).quantize_shared(bits)
+    check_shared_codes(layer_gpu, layer_or)
+    for T in (1, 160):
+        rep = check_forward(mote, layer_gpu, layer_or, synth.tokens(wl.with_T(T)))
+        assert rep["rel_fro"] < 5e-3

@@ -33,13 +33,15 @@ def test_rms_norm(mote, T, d):
     assert err <= REL_FRO_TOL
 
 
-@pytest.mark.parametrize("rms_eps", [1e-6, 0.0])
+@pytest.mark.parametrize("rms_eps,shared_bits", [(1e-6, 16), (0.0, 16), (1e-6, 8), (1e-6, 4)])
 @pytest.mark.parametrize("T", [1, 40, 150])          # decode path (1, 40) and tensor-core path (150)
-def test_small_stack_per_layer_parity(mote, T, rms_eps):
+def test_small_stack_per_layer_parity(mote, T, rms_eps, shared_bits):
     n_layers = 5
     wl = synth.custom("stack", 128, 256, 4, 2, T, 4100, n_layers=n_layers, w_std=0.08)
     masters = [synth.master_layer(wl, layer=l) for l in range(n_layers)]
     layers = [mote.MoteLayer.from_master(m) for m in masters]
+    if shared_bits != 16:                             # Section 4.3: RTN-coded shared experts
+        layers = [l.quantize_shared(shared_bits) for l in layers]
     stack = mote.MoteStack(layers)
     x_bits = synth.tokens(wl)
     x = bf16_tensor(x_bits)
@@ -57,6 +59,8 @@ def test_small_stack_per_layer_parity(mote, T, rms_eps):
     # every layer against the oracle, on the GPU's own input and residual of that layer
     for l in range(n_layers):
         layer_or = O.build_layer(masters[l])
+        if shared_bits != 16:
+            layer_or = O.quantize_shared(layer_or, shared_bits)
         res = taps[l].contiguous()
         xin_t = norm(res)
         got_t = taps[l + 1] if l + 1 < n_layers else out
