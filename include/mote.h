@@ -210,6 +210,11 @@ typedef struct {
 
 /* Bytes of scratch mote_moe_forward needs for up to T_max tokens (0 if the shape is invalid). */
 size_t mote_workspace_bytes(int d, int f, int E, int k, int64_t T_max);
+/* The same for one layer description.  Larger than mote_workspace_bytes only for an RTN-coded shared
+ * expert and T_max >= 768: 6*d*f more bytes, in which a prefill expands the shared expert's codes to
+ * bf16 once per call (a streaming pass) instead of expanding them inside the GEMM for every row
+ * tile.  A call that is given only mote_workspace_bytes() still runs, expanding inside the GEMM. */
+size_t mote_layer_workspace_bytes(const mote_layer_t* L, int64_t T_max);
 
 /* ------------------------------------------------------------------------------------------------
  * mote_moe_forward -- the whole layer (Eq. 2-8): route, dispatch, Q_a(x), gate/up ternary GEMM
@@ -237,7 +242,7 @@ mote_status_t mote_moe_forward(const mote_layer_t* L, const void* x_bf16,
 /* Same layer with HOST input and output: copies x_host (and residual_host if non-NULL) to the
  * device, runs mote_moe_forward, copies the result to out_host and waits for the stream.  Host
  * buffers should be page-locked for the copies to be asynchronous.  Needs
- * mote_workspace_bytes(...) + mote_host_staging_bytes(d, T) bytes of device scratch. */
+ * mote_layer_workspace_bytes(...) + mote_host_staging_bytes(d, T) bytes of device scratch. */
 size_t mote_host_staging_bytes(int d, int64_t T_max);
 mote_status_t mote_moe_forward_host(const mote_layer_t* L, const void* x_host,
                                     const void* residual_host, int64_t T, void* out_host,

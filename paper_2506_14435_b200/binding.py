@@ -57,6 +57,8 @@ lib.mote_route_topk.argtypes = [C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.
                                 C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
 lib.mote_workspace_bytes.restype = C.c_size_t
 lib.mote_workspace_bytes.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, C.c_int64]
+lib.mote_layer_workspace_bytes.restype = C.c_size_t
+lib.mote_layer_workspace_bytes.argtypes = [C.POINTER(mote_layer_t), C.c_int64]
 lib.mote_host_staging_bytes.restype = C.c_size_t
 lib.mote_host_staging_bytes.argtypes = [C.c_int, C.c_int64]
 lib.mote_moe_forward.restype = C.c_int
@@ -258,9 +260,9 @@ class MoteLayer:
         return s
 
     def workspace(self, T: int, host_staging: bool = False) -> torch.Tensor:
-        need = lib.mote_workspace_bytes(self.d, self.f, self.E, self.k, T)
+        need = lib.mote_layer_workspace_bytes(C.byref(self.struct()), T)
         if need == 0:
-            raise MoteError(2, "mote_workspace_bytes")
+            raise MoteError(2, "mote_layer_workspace_bytes")
         if host_staging:
             need += lib.mote_host_staging_bytes(self.d, T)
         if self._ws is None or self._ws.numel() < need:

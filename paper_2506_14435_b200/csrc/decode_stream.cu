@@ -16,8 +16,8 @@
 //                     (Eq. 3); the last CTA to finish builds the dispatch tables
 //   decode_gateup     routed gate/up (Eq. 6) + shared gate/up (Eq. 2): h, row maxima of h, h_shared
 //   (Q_a(h): quant_rows_known_beta_kernel of quant_act.cu)
-//   decode_down       routed down (Eq. 5) + shared down: y, s
-//   (combine: combine_kernel)
+//   decode_down       routed down (Eq. 5) + shared down: y, s; the CTA that finishes the last item
+//                     of a 16-column tile combines it (Eq. 2, Eq. 4) and writes the layer output
 #include <algorithm>
 
 #include "mote_common.cuh"
@@ -670,6 +670,12 @@ struct DecodeDownArgs {
   float* y;                     // [P, d]
   float* s;                     // [T, d]
   int32_t* tap_down;            // optional [P, d]
+  // combine of Eq. 2 / Eq. 4, done per 16-column tile by the CTA that finishes the tile's last item
+  const float* topk_w;          // [T, k]
+  const int32_t* perm;          // [T*k] pair -> sorted row
+  const uint16_t* residual;     // [T, d] bf16 or null; may alias out
+  uint16_t* out;                // [T, d] bf16
+  uint32_t* tile_count;         // [d/16] zero on entry
 };
 
 constexpr int kDownWarps = 16;
@@ -769,9 +775,38 @@ __device__ __forceinline__ void down_shared_tile(const DecodeDownArgs& a, int ti
   __syncthreads();
 }
 
+// The CTA that completes the last of a tile's items (the shared expert's and one per expert that
+// received tokens) adds them up: out[t, c] = bf16( s[t, c] + sum_j w[t, j] * y[perm[t*k+j], c] [+ residual] ),
+// fp32, slots in ascending j -- the arithmetic of combine_kernel.  Every thread calls this after
+// its stores of the item; the count is kept per tile, so the combines of different tiles run in
+// parallel on whichever CTAs arrive last.
+__device__ __forceinline__ void down_tile_done(const DecodeDownArgs& a, int tile, int n_producers, int* s_last) {
+  __threadfence();                                   // this thread's y / s values are visible device-wide
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const uint32_t old = atomicAdd(a.tile_count + tile, 1u);
+    *s_last = (old == (uint32_t)n_producers - 1u);
+    if (*s_last) a.tile_count[tile] = 0u;            // left clean for the next call
+  }
+  __syncthreads();
+  if (!*s_last) return;
+  __threadfence();
+  const int d = a.c.d, k = a.c.k, T = a.c.T;
+  for (int i = threadIdx.x; i < T * 16; i += blockDim.x) {
+    const int t = i >> 4, col = tile * 16 + (i & 15);
+    float acc = __ldcg(a.s + int64_t(t) * d + col);
+    for (int j = 0; j < k; ++j)
+      acc = fmaf(a.topk_w[t * k + j], __ldcg(a.y + int64_t(a.perm[t * k + j]) * d + col), acc);
+    if (a.residual) acc += __uint_as_float(uint32_t(a.residual[int64_t(t) * d + col]) << 16);
+    a.out[int64_t(t) * d + col] = (uint16_t)f32_to_bf16_bits(acc);
+  }
+  __syncthreads();
+}
+
 template <int NTB>
 __global__ void __launch_bounds__(kDownWarps * 32) decode_down_kernel(DecodeDownArgs a) {
   __shared__ ExpertList s_list;
+  __shared__ int s_last;
   extern __shared__ float s_part[];                       // kDownWarps * NTB * 4 * 32 floats
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // This kernel is let in as soon as Q_a(h) has STARTED (which is after the gate/up kernel and
@@ -791,6 +826,7 @@ __global__ void __launch_bounds__(kDownWarps * 32) decode_down_kernel(DecodeDown
     }
     if (item < n_shared) {
       down_shared_tile<NTB>(a, item, warp, lane, s_part);
+      down_tile_done(a, item, 1 + s_list.n, &s_last);
     } else {
       const int r = item - n_shared;
       const int e = s_list.id[r / tiles];
@@ -800,6 +836,7 @@ __global__ void __launch_bounds__(kDownWarps * 32) decode_down_kernel(DecodeDown
       else if (NTB == 2 || nt <= 2) down_routed_tile<(NTB >= 2 ? 2 : 1)>(a, e, tile, warp, lane, ip);
       else if (NTB == 4 || nt <= 4) down_routed_tile<(NTB >= 4 ? 4 : 1)>(a, e, tile, warp, lane, ip);
       else down_routed_tile<(NTB >= 8 ? 8 : 1)>(a, e, tile, warp, lane, ip);
+      down_tile_done(a, tile, 1 + s_list.n, &s_last);
     }
   }
   if (!waited) pdl_wait();                 // no CTA leaves before the kernels ahead of it are complete
@@ -868,6 +905,8 @@ mote_status_t launch_decode_stream(const DecodeStreamArgs& p, int phase, cudaStr
 
   DecodeDownArgs da{};
   da.c = c; da.down_packed = p.down_packed; da.alpha_down = p.alpha_down;
+  da.topk_w = p.topk_w; da.perm = p.perm; da.residual = static_cast<const uint16_t*>(p.residual);
+  da.out = static_cast<uint16_t*>(p.out); da.tile_count = p.tile_count;
   da.sh_down = p.sh_down; da.sh_bits = p.shared_bits; da.qh = p.qh; da.beta_h = p.beta_h; da.rowsum_h = p.rowsum_h;
   da.hs = static_cast<const uint16_t*>(p.hs); da.y = p.y; da.s = p.s; da.tap_down = p.tap_down;
   const int tiles = d / 16;

@@ -23,18 +23,30 @@ static inline void stage_mark(int i, cudaStream_t stream) {
   if (g_timer.active) cudaEventRecord(g_timer.ev[i], stream);
 }
 
+// Head of the workspace, cleared at the start of every call: [0] device status word, [1] arrival
+// counter of the decode prologue, from byte 256 on the per-tile arrival counters of the decode
+// path's down kernel (d / 16 <= 2048 words).
+constexpr size_t kStatusBytes = 256 + 2048 * 4;
+
 struct Plan {
   size_t status, topk_idx, topk_w, offsets, perm, inv;
   size_t qx, beta_x, rowsum_x, h, qh, beta_h, rowsum_h, y, hs, s, tiles_routed, tiles_shared, blk_hist, blk_base;
   size_t total;
+  size_t sh_codes_bf16;   // the three RTN-coded shared matrices expanded to bf16 (prefill); after `total`
+  size_t total_expanded;
 };
+
+// From this many tokens on, a prefill with an RTN-coded shared expert first expands the codes of the
+// layer to bf16 in the workspace (one streaming pass) and runs the plain bf16 GEMMs on them; below,
+// the GEMM expands the codes tile by tile in shared memory (less weight traffic, more work per row tile).
+constexpr int64_t kExpandMinTokens = 768;
 
 static Plan make_plan(int d, int f, int E, int k, int64_t T) {
   Plan p{};
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off += round_up(std::max<size_t>(bytes, 1), 256); return o; };
   const size_t P = size_t(T) * k;
-  p.status = take(256);
+  p.status = take(kStatusBytes);
   p.topk_idx = take(P * 4);
   p.topk_w = take(P * 4);
   p.offsets = take(size_t(E + 1) * 4);
@@ -56,7 +68,45 @@ static Plan make_plan(int d, int f, int E, int k, int64_t T) {
   p.blk_hist = take(n_blk * E * 4);
   p.blk_base = take(n_blk * E * 4);
   p.total = off;
+  p.sh_codes_bf16 = take(T >= kExpandMinTokens ? size_t(3) * d * f * 2 : 1);
+  p.total_expanded = T >= kExpandMinTokens ? off : p.total;
   return p;
+}
+
+// RTN codes (int8, or 4-bit in the pair-split word order) -> the same integers as bf16, 16 code
+// bytes per thread and step.
+struct ExpandArgs { const uint4* codes[3]; uint4* out[3]; };
+__global__ void __launch_bounds__(256) expand_codes_kernel(ExpandArgs a, int64_t n_chunks, int bits) {
+  const uint4* __restrict__ codes = a.codes[blockIdx.y];     // blockIdx.y: gate, up, down
+  uint4* __restrict__ out = a.out[blockIdx.y];
+  const int64_t stride = int64_t(gridDim.x) * blockDim.x;
+  for (int64_t i = int64_t(blockIdx.x) * blockDim.x + threadIdx.x; i < n_chunks; i += stride) {
+    const uint4 w = codes[i];
+    const uint32_t pw[4] = {w.x, w.y, w.z, w.w};
+    if (bits == 8) {
+      uint32_t e[8];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) s8x4_to_bf16x2(pw[j], e[2 * j], e[2 * j + 1]);
+      out[2 * i] = make_uint4(e[0], e[1], e[2], e[3]);
+      out[2 * i + 1] = make_uint4(e[4], e[5], e[6], e[7]);
+    } else {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        uint32_t e[4];
+        u4x8_to_bf16x2(pw[j], e);
+        out[4 * i + j] = make_uint4(e[0], e[1], e[2], e[3]);
+      }
+    }
+  }
+}
+
+static mote_status_t launch_expand_codes(const ExpandArgs& a, int64_t elements, int bits, cudaStream_t stream) {
+  const int64_t n_chunks = elements / (bits == 8 ? 16 : 32);
+  const unsigned grid = (unsigned)std::min<int64_t>((n_chunks + 255) / 256, 148 * 8);
+  expand_codes_kernel<<<dim3(grid, 3), 256, 0, stream>>>(a, n_chunks, bits);
+  ++g_launch_count;
+  MOTE_LAUNCH_OK();
+  return MOTE_OK;
 }
 
 static bool shape_ok(int d, int f, int E, int k) {
@@ -116,6 +166,13 @@ extern "C" const char* mote_status_string(mote_status_t st) {
 extern "C" size_t mote_workspace_bytes(int d, int f, int E, int k, int64_t T_max) {
   if (!shape_ok(d, f, E, k) || T_max < 0 || T_max > (int64_t(1) << 24)) return 0;
   return make_plan(d, f, E, k, T_max).total;
+}
+
+extern "C" size_t mote_layer_workspace_bytes(const mote_layer_t* L, int64_t T_max) {
+  if (!L || !shape_ok(L->d, L->f, L->E, L->k) || T_max < 0 || T_max > (int64_t(1) << 24)) return 0;
+  const Plan pl = make_plan(L->d, L->f, L->E, L->k, T_max);
+  const bool rtn = L->shared_bits == MOTE_SHARED_INT8 || L->shared_bits == MOTE_SHARED_INT4;
+  return rtn ? pl.total_expanded : pl.total;
 }
 
 extern "C" size_t mote_host_staging_bytes(int d, int64_t T_max) {
@@ -202,8 +259,8 @@ extern "C" mote_status_t mote_moe_forward(const mote_layer_t* L, const void* x, 
   const int interleave = (tensor || path == MOTE_PATH_STREAM) ? 1 : 0;
 
   if (path == MOTE_PATH_STREAM) {
-    // status word and the prologue's arrival counter
-    MOTE_CUDA_OK(cudaMemsetAsync(status, 0, 8, stream));
+    // status word, the prologue's arrival counter, the down kernel's tile counters
+    MOTE_CUDA_OK(cudaMemsetAsync(status, 0, 256 + size_t(d / 16) * 4, stream));
     stage_mark(0, stream);
     DecodeStreamArgs ds{};
     ds.x = x; ds.T = T; ds.d = d; ds.f = f; ds.E = E; ds.k = k; ds.norm_topk = L->norm_topk;
@@ -214,6 +271,7 @@ extern "C" mote_status_t mote_moe_forward(const mote_layer_t* L, const void* x, 
     ds.topk_idx = topk_idx; ds.topk_w = topk_w; ds.offsets = offsets; ds.perm = perm; ds.inv = inv;
     ds.qx = qx; ds.beta_x = beta_x; ds.rowsum_x = rowsum_x; ds.h = h; ds.qh = qh; ds.beta_h = beta_h;
     ds.rowsum_h = rowsum_h; ds.y = y; ds.hs = hs; ds.s = s; ds.counter = status + 1;
+    ds.tile_count = status + 64; ds.residual = residual; ds.out = out;
     ds.tap_gate = taps ? taps->acc_gate : nullptr; ds.tap_up = taps ? taps->acc_up : nullptr;
     ds.tap_down = taps ? taps->acc_down : nullptr;
     if (taps && (!taps->acc_gate != !taps->acc_up)) return MOTE_ERR_NULL;
@@ -226,12 +284,9 @@ extern "C" mote_status_t mote_moe_forward(const mote_layer_t* L, const void* x, 
     st = launch_quant_rows_known_beta(h, P, f, qh, beta_h, rowsum_h, 1, stream, true, true);
     if (st) return st;
     stage_mark(5, stream);
-    st = launch_decode_stream(ds, 2, stream);                 // routed and shared down
+    st = launch_decode_stream(ds, 2, stream);                 // routed and shared down, combine
     if (st) return st;
-    stage_mark(6, stream); stage_mark(7, stream); stage_mark(8, stream);
-    st = launch_combine(s, y, topk_w, perm, residual, T, d, k, out, stream, true);
-    if (st) return st;
-    stage_mark(9, stream);
+    stage_mark(6, stream); stage_mark(7, stream); stage_mark(8, stream); stage_mark(9, stream);
     if (taps) {
       auto d2d = [&](void* dst, const void* src, size_t bytes) -> bool {
         return !dst || cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToDevice, stream) == cudaSuccess;
@@ -256,6 +311,22 @@ extern "C" mote_status_t mote_moe_forward(const mote_layer_t* L, const void* x, 
 
   mote_status_t st;
   MOTE_CUDA_OK(cudaMemsetAsync(status, 0, 4, stream));
+  // prefill with an RTN-coded shared expert and room in the workspace: expand the codes to bf16 once
+  SharedMat xg = sh_gate, xu = sh_up, xd = sh_down;
+  int x_bits = sh_bits;
+  if (sh_rtn && tensor && T >= kExpandMinTokens && ws_bytes >= pl.total_expanded) {
+    char* e0 = base + pl.sh_codes_bf16;
+    const size_t mat = size_t(d) * f * 2;
+    ExpandArgs ea{};
+    for (int i = 0; i < 3; ++i) {
+      ea.codes[i] = static_cast<const uint4*>(i == 0 ? sh_gate.w : i == 1 ? sh_up.w : sh_down.w);
+      ea.out[i] = reinterpret_cast<uint4*>(e0 + i * mat);
+    }
+    st = launch_expand_codes(ea, int64_t(d) * f, sh_bits, stream);
+    if (st) return st;
+    xg.w = e0; xu.w = e0 + mat; xd.w = e0 + 2 * mat;
+    x_bits = MOTE_SHARED_BF16;                     // bf16 operands; the row scales still apply
+  }
   stage_mark(0, stream);
   // S1 router, S2 dispatch
   // block-wise dispatch: the tensor-core router (d % 32 == 0) leaves per-block expert counts, a small
@@ -314,7 +385,7 @@ extern "C" mote_status_t mote_moe_forward(const mote_layer_t* L, const void* x, 
   if (st) return st;
   stage_mark(6, stream);
   // S7 shared expert
-  st = tensor ? launch_shared_umma(x, sh_gate, sh_up, sh_bits, true, T, d, f, hs, tiles_shared, max_mtiles_shared,
+  st = tensor ? launch_shared_umma(x, xg, xu, x_bits, true, T, d, f, hs, tiles_shared, max_mtiles_shared,
                                    status, nullptr, stream, pdl)
               : launch_shared_gateup_simt(x, sh_gate, sh_up, sh_bits, T, d, f, hs, stream);
   if (st) return st;
@@ -323,7 +394,7 @@ extern "C" mote_status_t mote_moe_forward(const mote_layer_t* L, const void* x, 
     // shared down projection with S8 (combine, residual, bf16 rounding) in its epilogue; the fp32
     // shared output is written only when a tap asks for it
     CombineArgs cb{y, topk_w, perm, residual, out, k};
-    st = launch_shared_umma(hs, sh_down, SharedMat{nullptr, nullptr}, sh_bits, false, T, f, d,
+    st = launch_shared_umma(hs, xd, SharedMat{nullptr, nullptr}, x_bits, false, T, f, d,
                             (taps && taps->shared_out) ? s : nullptr, tiles_shared, max_mtiles_shared, status, &cb,
                             stream, pdl);
     if (st) return st;
@@ -367,7 +438,7 @@ extern "C" size_t mote_stack_workspace_bytes(const mote_layer_t* layers, int n_l
   if (!layers || n_layers < 1 || T_max < 0) return 0;
   size_t core = 0;
   for (int l = 0; l < n_layers; ++l) {
-    const size_t b = mote_workspace_bytes(layers[l].d, layers[l].f, layers[l].E, layers[l].k, T_max);
+    const size_t b = mote_layer_workspace_bytes(&layers[l], T_max);
     if (b == 0 || layers[l].d != layers[0].d) return 0;
     core = std::max(core, b);
   }
@@ -422,7 +493,7 @@ extern "C" mote_status_t mote_moe_forward_host(const mote_layer_t* L, const void
   if (T < 0) return MOTE_ERR_SHAPE;
   if (T == 0) return MOTE_OK;
   if (!x_host || !out_host || !ws) return MOTE_ERR_NULL;
-  const size_t core = mote_workspace_bytes(L->d, L->f, L->E, L->k, T);
+  const size_t core = mote_layer_workspace_bytes(L, T);
   if (core == 0) return MOTE_ERR_SHAPE;
   const size_t slab = round_up(size_t(T) * L->d * 2, 256);
   if (ws_bytes < core + 3 * slab) return MOTE_ERR_WORKSPACE;

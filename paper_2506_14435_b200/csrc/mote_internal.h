@@ -102,8 +102,8 @@ mote_status_t launch_shared_down_simt(const void* h, const SharedMat& Wd, int bi
                                       cudaStream_t stream);
 
 // Decode path (T <= 64): prologue (Q_a(x), router, dispatch), streamed gate/up, Q_a(h), streamed
-// down.  Fills topk_*, offsets/perm/inv, qx (TOKEN order, k-interleaved), beta_x/rowsum_x (token
-// order), h, beta_h, qh, rowsum_h, y, hs, s; the caller runs the combine.
+// down with the combine.  Fills topk_*, offsets/perm/inv, qx (TOKEN order, k-interleaved),
+// beta_x/rowsum_x (token order), h, beta_h, qh, rowsum_h, y, hs, s and the layer output.
 struct DecodeStreamArgs {
   const void* x; int64_t T; int d, f, E, k, norm_topk;
   const float* Wr; const float* router_bias;
@@ -114,6 +114,8 @@ struct DecodeStreamArgs {
   int8_t* qx; float* beta_x; int32_t* rowsum_x;
   void* h; int8_t* qh; float* beta_h; int32_t* rowsum_h; float* y; void* hs; float* s;
   uint32_t* counter;                       // one zeroed word
+  uint32_t* tile_count;                    // d/16 zeroed words
+  const void* residual; void* out;         // [T, d] bf16 (residual may be null, may alias out)
   int32_t* tap_gate; int32_t* tap_up; int32_t* tap_down;   // optional
 };
 bool decode_stream_supported(int d, int f, int E, int k, int64_t T);

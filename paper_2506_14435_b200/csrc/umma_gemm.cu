@@ -281,36 +281,47 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
             if (!ok) break;
             const uint8_t* src = genP + pstage * TR::kStageP;
             uint8_t* dst = genB + stage * kStageB;
-            for (int c = tid; c < n_chunks; c += 128) {
-              const uint4 w = *reinterpret_cast<const uint4*>(src + c * 16);
-              const uint32_t pw[4] = {w.x, w.y, w.z, w.w};
-              if (TR::kRtnBits == 8) {
-                // 16 int8 codes -> two 16-byte pieces of 8 bf16 each
-                const int r = c >> 2, quarter = c & 3;
-                uint8_t* row = dst + (r >> 3) * 1024 + (r & 7) * 128;
-                uint32_t e[8];
+            // batches of four chunks per thread, all loads of a batch ahead of its conversions
+            for (int c0 = tid; c0 < n_chunks; c0 += 128 * 4) {
+              uint4 wv[4];
 #pragma unroll
-                for (int j = 0; j < 4; ++j) s8x4_to_bf16x2(pw[j], e[2 * j], e[2 * j + 1]);
-                *reinterpret_cast<uint4*>(row + (((quarter * 2) ^ (r & 7)) << 4)) = make_uint4(e[0], e[1], e[2], e[3]);
-                *reinterpret_cast<uint4*>(row + (((quarter * 2 + 1) ^ (r & 7)) << 4)) = make_uint4(e[4], e[5], e[6], e[7]);
-              } else {
-                const int r = c >> 1, half = c & 1;
-                uint8_t* row = dst + (r >> 3) * 1024 + (r & 7) * 128;
+              for (int b = 0; b < 4; ++b) {
+                const int c = c0 + b * 128;
+                if (c < n_chunks) wv[b] = *reinterpret_cast<const uint4*>(src + c * 16);
+              }
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                  uint4 o;
-                  if (TR::kRtnBits == 4) {
-                    // 8 four-bit codes -> one 16-byte piece of 8 bf16
-                    uint32_t e[4];
-                    u4x8_to_bf16x2(pw[j], e);
-                    o = make_uint4(e[0], e[1], e[2], e[3]);
-                  } else {
-                    o.x = pw[j] & 0x03030303u;
-                    o.y = (pw[j] >> 2) & 0x03030303u;
-                    o.z = (pw[j] >> 4) & 0x03030303u;
-                    o.w = (pw[j] >> 6) & 0x03030303u;
+              for (int b = 0; b < 4; ++b) {
+                const int c = c0 + b * 128;
+                if (c >= n_chunks) break;
+                const uint32_t pw[4] = {wv[b].x, wv[b].y, wv[b].z, wv[b].w};
+                if (TR::kRtnBits == 8) {
+                  // 16 int8 codes -> two 16-byte pieces of 8 bf16 each
+                  const int r = c >> 2, quarter = c & 3;
+                  uint8_t* row = dst + (r >> 3) * 1024 + (r & 7) * 128;
+                  uint32_t e[8];
+#pragma unroll
+                  for (int j = 0; j < 4; ++j) s8x4_to_bf16x2(pw[j], e[2 * j], e[2 * j + 1]);
+                  *reinterpret_cast<uint4*>(row + (((quarter * 2) ^ (r & 7)) << 4)) = make_uint4(e[0], e[1], e[2], e[3]);
+                  *reinterpret_cast<uint4*>(row + (((quarter * 2 + 1) ^ (r & 7)) << 4)) = make_uint4(e[4], e[5], e[6], e[7]);
+                } else {
+                  const int r = c >> 1, half = c & 1;
+                  uint8_t* row = dst + (r >> 3) * 1024 + (r & 7) * 128;
+#pragma unroll
+                  for (int j = 0; j < 4; ++j) {
+                    uint4 o;
+                    if (TR::kRtnBits == 4) {
+                      // 8 four-bit codes -> one 16-byte piece of 8 bf16
+                      uint32_t e[4];
+                      u4x8_to_bf16x2(pw[j], e);
+                      o = make_uint4(e[0], e[1], e[2], e[3]);
+                    } else {
+                      o.x = pw[j] & 0x03030303u;
+                      o.y = (pw[j] >> 2) & 0x03030303u;
+                      o.z = (pw[j] >> 4) & 0x03030303u;
+                      o.w = (pw[j] >> 6) & 0x03030303u;
+                    }
+                    *reinterpret_cast<uint4*>(row + (((half * 4 + j) ^ (r & 7)) << 4)) = o;
                   }
-                  *reinterpret_cast<uint4*>(row + (((half * 4 + j) ^ (r & 7)) << 4)) = o;
                 }
               }
             }
@@ -386,8 +397,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
                 }
 #pragma unroll
                 for (int j = 0; j < 16; ++j) hmax = fmaxf(hmax, fabsf(hv[j]));
-              } else if (TR::kRtn) {
-                // row scales of the gate and up matrices = scales of this tile's output columns
+              } else if (TR::kRtn || a.alpha0 != nullptr) {
+                // RTN-coded shared expert (codes expanded here, or beforehand): row scales of the
+                // gate and up matrices = scales of this tile's output columns
                 const float4* sgp = reinterpret_cast<const float4*>(a.alpha0 + col0 + c);
                 const float4* sup = reinterpret_cast<const float4*>(a.alpha1 + col0 + c);
 #pragma unroll
@@ -474,7 +486,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
 #pragma unroll
             for (int v = 0; v < 16; ++v)
               o[v] = TR::kTernary ? __fmul_rn(i2f_small((int)ra[v] - rs), c0) : __uint_as_float(ra[v]);
-            if (TR::kRtn) {
+            if (TR::kRtn || (!TR::kTernary && a.alpha0 != nullptr)) {
               const float4* sp = reinterpret_cast<const float4*>(a.alpha0 + col0 + c);
 #pragma unroll
               for (int v = 0; v < 4; ++v) {
@@ -678,7 +690,7 @@ mote_status_t launch_shared_umma(const void* act, const SharedMat& w0, const Sha
   a.b_rows_per_expert = 0;
   a.out = out;
   a.status = status;
-  a.alpha0 = w0.scale; a.alpha1 = w1.scale;     // RTN modes only
+  a.alpha0 = w0.scale; a.alpha1 = w1.scale;     // row scales of an RTN-coded shared expert, else null
   if (comb && !gateup) {
     a.comb_y = comb->y; a.comb_w = comb->w; a.comb_perm = comb->perm;
     a.comb_res = static_cast<const uint16_t*>(comb->residual); a.comb_out = static_cast<uint16_t*>(comb->out);

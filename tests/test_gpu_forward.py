@@ -166,6 +166,7 @@ def test_host_buffer_entry_point(mote):
     (128, 384, 4, 1, 130, dict(norm_topk=0), TENSOR),     # down projection with 128-wide tiles
     (384, 640, 3, 3, 515, {}, TENSOR),                    # several row tiles, 160-wide down tiles (128 + 32 rows)
     (896, 4864, 4, 2, 160, dict(outlier_frac=0.01), TENSOR),  # 224-wide down tiles
+    (256, 512, 4, 2, 900, {}, TENSOR),                    # long enough for the codes to be expanded once per call
     (64, 128, 3, 3, 5, {}, STREAM),                       # one short reduction step (32 bytes of 4-bit codes)
     (128, 192, 2, 1, 1, {}, STREAM),
     (896, 4864, 4, 2, 17, dict(outlier_frac=0.01), STREAM),
@@ -204,3 +205,26 @@ def test_rtn_shared_expert_rejects_missing_scales(mote):
     with pytest.raises(mote.MoteError) as ei:
         mote.mote_moe_forward(layer_gpu, bf16_tensor(synth.tokens(wl)))
     assert ei.value.status == 2
+
+
+@pytest.mark.parametrize("bits", [8, 4])
+def test_rtn_prefill_expanding_once_or_inside_the_gemm_agree(mote, bits):
+    # with only mote_workspace_bytes() of scratch a long prefill expands the codes inside the GEMM;
+    # with mote_layer_workspace_bytes() it expands them once: same integers, same sums
+    import ctypes as C
+    wl = synth.custom("rtn", 256, 512, 4, 2, 900, 4321)
+    master, layer_or, layer_gpu = _setup(mote, wl, TENSOR)
+    layer_q = layer_gpu.quantize_shared(bits)
+    x = bf16_tensor(synth.tokens(wl))
+    small = mote.lib.mote_workspace_bytes(wl.d, wl.f, wl.E, wl.k, wl.T)
+    s = layer_q.struct()
+    assert mote.lib.mote_layer_workspace_bytes(C.byref(s), wl.T) == small + 6 * wl.d * wl.f
+    assert mote.lib.mote_layer_workspace_bytes(C.byref(layer_gpu.struct()), wl.T) == small
+    ws = torch.empty(small, dtype=torch.uint8, device="cuda")
+    out1 = torch.empty_like(x)
+    st = mote.lib.mote_moe_forward(C.byref(s), x.data_ptr(), None, wl.T, out1.data_ptr(), None, ws.data_ptr(), small,
+                                   C.c_void_p(torch.cuda.current_stream().cuda_stream))
+    assert st == 0
+    out2 = mote.mote_moe_forward(layer_q, x)
+    torch.cuda.synchronize()
+    assert torch.equal(out1, out2)
