@@ -170,6 +170,23 @@ def router(x_bf16, Wr, bias, k: int, norm_topk: int):
     return dict(logits=logits, idx=idx, w=w, near_tie=near_tie)
 
 
+def load_balance_stats(logits: np.ndarray, idx: np.ndarray, E: int):
+    """The two per-expert factors of the load-balancing loss (Eq. 12) for a batch of tokens:
+    t_i = number of (token, slot) pairs routed to expert i, and sum_x P(x)_i, the routing
+    probabilities of Eq. 3 (softmax over all E experts) summed over the batch.  fp64."""
+    logits = np.asarray(logits, dtype=np.float64)
+    ex = np.exp(logits - logits.max(axis=1, keepdims=True))
+    P = ex / ex.sum(axis=1, keepdims=True)
+    t = np.bincount(np.asarray(idx).ravel(), minlength=E).astype(np.int64)
+    return t, P.sum(axis=0)
+
+
+def balance_loss(t: np.ndarray, prob_sum: np.ndarray, n_tokens: int) -> float:
+    """Eq. 12 as printed: L_balance = E / |X| * sum_i t_i * sum_x P(x)_i."""
+    E = len(t)
+    return float(E) / float(n_tokens) * float(np.sum(np.asarray(t, np.float64) * np.asarray(prob_sum, np.float64)))
+
+
 def dispatch(idx: np.ndarray, E: int):
     """Group the T*k (token, slot) pairs by expert, keeping (token, slot) order inside each
     expert (a stable counting sort).  pair p = t*k + j.

@@ -353,3 +353,28 @@ def test_int4_storage_by_hand_and_size():
     # bytes per weight behind the Table 3 footprints: 1 (INT8) and 1/2 (INT4), scales not counted
     q8, _ = O.rtn_quantize(rng.standard_normal((16, 64)).astype(np.float32), 8)
     assert q8.nbytes == 16 * 64 and packed.nbytes * 2 == q.size
+
+
+# ------------------------------------------------------------------ Eq. 12: load-balance factors
+def test_load_balance_stats_and_loss():
+    rng = np.random.default_rng(80)
+    T, E, k = 57, 6, 2
+    logits = rng.standard_normal((T, E)) * 2
+    idx = np.argsort(-logits, axis=1, kind="stable")[:, :k]
+    t, S = O.load_balance_stats(logits, idx, E)
+    assert t.sum() == T * k and math.isclose(S.sum(), T, rel_tol=1e-12)     # probabilities sum to 1 per token
+    # brute force
+    for i in range(E):
+        assert t[i] == sum(1 for tt in range(T) for j in range(k) if idx[tt, j] == i)
+        ref = sum(math.exp(logits[tt, i]) / sum(math.exp(v) for v in logits[tt]) for tt in range(T))
+        assert math.isclose(S[i], ref, rel_tol=1e-12)
+    assert np.allclose(S, torch.softmax(torch.from_numpy(logits), dim=1).sum(0).numpy(), rtol=1e-12)
+    # uniform router, top-1, perfectly balanced batch: t_i = T/E and sum_x P_i = T/E, so Eq. 12 gives T
+    T = 24
+    t, S = O.load_balance_stats(np.zeros((T, E)), (np.arange(T) % E)[:, None], E)
+    assert np.all(t == T // E) and np.allclose(S, T / E)
+    assert math.isclose(O.balance_loss(t, S, T), T, rel_tol=1e-12)
+    # everything routed to one expert that also holds all the probability: E times larger
+    lg = np.full((T, E), -1e3); lg[:, 2] = 0.0
+    t, S = O.load_balance_stats(lg, np.full((T, 1), 2), E)
+    assert math.isclose(O.balance_loss(t, S, T), E * T, rel_tol=1e-12)
