@@ -167,6 +167,19 @@ mote_status_t mote_route_topk(const void* x_bf16, int64_t T, int64_t d,
                               int32_t* topk_idx, float* topk_w, float* logits, void* stream);
 
 /* ------------------------------------------------------------------------------------------------
+ * mote_route_stats -- the two per-expert factors of the load-balancing loss (Eq. 12) for a batch,
+ * from the router's outputs:
+ *     tokens_per_expert[i] = t_i        number of (token, slot) pairs routed to expert i
+ *     prob_sum[i]          = sum_x P(x)_i   routing probability of Eq. 3 (softmax over all E experts)
+ * so that L_balance = E / T * sum_i t_i * prob_sum[i].  fp32, summed in a fixed order (reproducible).
+ *   logits [T,E] float (the optional output of mote_route_topk), topk_idx [T,k] int32,
+ *   tokens_per_expert [E] int32, prob_sum [E] float.  T = 0 gives zeros.
+ * Errors: E, k out of range -> ERR_SHAPE; NULL -> ERR_NULL.
+ */
+mote_status_t mote_route_stats(const float* logits, const int32_t* topk_idx, int64_t T, int E, int k,
+                               int32_t* tokens_per_expert, float* prob_sum, void* stream);
+
+/* ------------------------------------------------------------------------------------------------
  * Layer description (Eq. 2-6).  All device pointers, immutable while calls are in flight.
  */
 typedef struct {

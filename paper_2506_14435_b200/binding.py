@@ -55,6 +55,8 @@ lib.mote_quant_act.argtypes = [C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_
 lib.mote_route_topk.restype = C.c_int
 lib.mote_route_topk.argtypes = [C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.c_int, C.c_int,
                                 C.c_int, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+lib.mote_route_stats.restype = C.c_int
+lib.mote_route_stats.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
 lib.mote_workspace_bytes.restype = C.c_size_t
 lib.mote_workspace_bytes.argtypes = [C.c_int, C.c_int, C.c_int, C.c_int, C.c_int64]
 lib.mote_layer_workspace_bytes.restype = C.c_size_t
@@ -176,6 +178,18 @@ def mote_route_topk(x, Wr, bias, k: int, norm_topk: int = 1, want_logits: bool =
     _check(lib.mote_route_topk(_ptr(x), T, d, _ptr(Wr), _ptr(bias), E, k, norm_topk, _ptr(idx), _ptr(w),
                                _ptr(logits), _stream()), "mote_route_topk")
     return idx, w, logits
+
+
+def mote_route_stats(logits: torch.Tensor, topk_idx: torch.Tensor):
+    """Eq. 12: (tokens_per_expert int32[E], prob_sum f32[E]) of a routed batch."""
+    _need_cuda(logits, topk_idx)
+    T, E = logits.shape
+    k = topk_idx.shape[1]
+    cnt = torch.empty(E, dtype=torch.int32, device=logits.device)
+    ps = torch.empty(E, dtype=torch.float32, device=logits.device)
+    _check(lib.mote_route_stats(_ptr(logits), _ptr(topk_idx), T, E, k, _ptr(cnt), _ptr(ps), _stream()),
+           "mote_route_stats")
+    return cnt, ps
 
 
 class MoteLayer:

@@ -437,21 +437,21 @@ __device__ __forceinline__ void split_steps(int n_steps, int n_parts, int p, int
 
 // Two rows of one shared-expert matrix against the token columns: bf16 values or RTN codes.
 // K = reduction length in elements; warp `part` of `n_parts` takes its share of the steps.
-template <int NT>
-__device__ __forceinline__ void shared_rows(const void* W, int bits, int64_t row_a, int64_t row_b, int K,
+template <int NT, int kShBits>
+__device__ __forceinline__ void shared_rows(const void* W, int64_t row_a, int64_t row_b, int K,
                                             const uint16_t* const (&tok)[NT], int n_parts, int part, int lane,
                                             float (&acc)[NT][4]) {
   int sb, se;
-  if (bits == 16) {
+  if (kShBits == 16) {
     const uint16_t* w = static_cast<const uint16_t*>(W);
     split_steps(K / 32, n_parts, part, sb, se);
     bf16_rows_steps<NT>(w + row_a * K, w + row_b * K, tok, sb, se, lane, acc);
   } else {
     const uint8_t* w = static_cast<const uint8_t*>(W);
-    const int k_bytes = bits == 8 ? K : K / 2;
+    const int k_bytes = kShBits == 8 ? K : K / 2;
     split_steps((k_bytes + 63) / 64, n_parts, part, sb, se);
-    if (bits == 8) rtn_rows_steps<NT, 8>(w + row_a * k_bytes, w + row_b * k_bytes, tok, sb, se, k_bytes, lane, acc);
-    else rtn_rows_steps<NT, 4>(w + row_a * k_bytes, w + row_b * k_bytes, tok, sb, se, k_bytes, lane, acc);
+    rtn_rows_steps<NT, kShBits == 16 ? 8 : kShBits>(w + row_a * k_bytes, w + row_b * k_bytes, tok, sb, se, k_bytes,
+                                                    lane, acc);
   }
 }
 
@@ -559,7 +559,7 @@ __device__ __forceinline__ void gateup_routed_tile(const DecodeGateUpArgs& a, in
   }
 }
 
-template <int NT>
+template <int NT, int kShBits>
 __device__ __forceinline__ void gateup_shared_tile(const DecodeGateUpArgs& a, int tile, int warp, int lane,
                                                    float* s_part) {
   const int d = a.c.d, f = a.c.f, T = a.c.T;
@@ -572,19 +572,18 @@ __device__ __forceinline__ void gateup_shared_tile(const DecodeGateUpArgs& a, in
 #pragma unroll
   for (int n = 0; n < NT; ++n) acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.0f;
   // gate row in fragment rows 0-7, up row in 8-15: two different matrices, one call each half
-  if (a.sh_bits == 16) {
+  if (kShBits == 16) {
     int sb, se;
     split_steps(d / 32, kGuWarps, warp, sb, se);
     bf16_rows_steps<NT>(static_cast<const uint16_t*>(a.sh_gate.w) + int64_t(frow) * d,
                         static_cast<const uint16_t*>(a.sh_up.w) + int64_t(frow) * d, tok, sb, se, lane, acc);
   } else {
-    const int k_bytes = a.sh_bits == 8 ? d : d / 2;
+    const int k_bytes = kShBits == 8 ? d : d / 2;
     const uint8_t* rg = static_cast<const uint8_t*>(a.sh_gate.w) + int64_t(frow) * k_bytes;
     const uint8_t* ru = static_cast<const uint8_t*>(a.sh_up.w) + int64_t(frow) * k_bytes;
     int sb, se;
     split_steps((k_bytes + 63) / 64, kGuWarps, warp, sb, se);
-    if (a.sh_bits == 8) rtn_rows_steps<NT, 8>(rg, ru, tok, sb, se, k_bytes, lane, acc);
-    else rtn_rows_steps<NT, 4>(rg, ru, tok, sb, se, k_bytes, lane, acc);
+    rtn_rows_steps<NT, kShBits == 16 ? 8 : kShBits>(rg, ru, tok, sb, se, k_bytes, lane, acc);
   }
   // partial sums of the 4 warps are added in warp order
 #pragma unroll
@@ -592,8 +591,8 @@ __device__ __forceinline__ void gateup_shared_tile(const DecodeGateUpArgs& a, in
 #pragma unroll
     for (int i = 0; i < 4; ++i) s_part[(warp * NT * 4 + n * 4 + i) * 32 + lane] = acc[n][i];
   __syncthreads();
-  const float sc_g = a.sh_bits == 16 ? 1.0f : a.sh_gate.scale[frow];
-  const float sc_u = a.sh_bits == 16 ? 1.0f : a.sh_up.scale[frow];
+  const float sc_g = kShBits == 16 ? 1.0f : a.sh_gate.scale[frow];
+  const float sc_u = kShBits == 16 ? 1.0f : a.sh_up.scale[frow];
   for (int n = warp; n < NT; n += kGuWarps) {
     float v[4];
 #pragma unroll
@@ -617,7 +616,9 @@ __device__ __forceinline__ void gateup_shared_tile(const DecodeGateUpArgs& a, in
 }
 
 // NTB = number of 8-token column tiles the launch is built for (1, 2, 4 or 8): ceil(T / 8) rounded up
-template <int NTB>
+// kShBits = storage of the shared expert (16, 8 or 4): a kernel of its own per width, so that the
+// code expansion of the RTN widths costs the bf16 kernel no registers
+template <int NTB, int kShBits>
 __global__ void __launch_bounds__(kGuWarps * 32) decode_gateup_kernel(DecodeGateUpArgs a) {
   __shared__ ExpertList s_list;
   __shared__ float s_part[kGuWarps * NTB * 4 * 32];
@@ -639,7 +640,7 @@ __global__ void __launch_bounds__(kGuWarps * 32) decode_gateup_kernel(DecodeGate
     }
     if (item >= n_items) break;
     if (item < n_shared) {
-      gateup_shared_tile<NTB>(a, item, warp, lane, s_part);
+      gateup_shared_tile<NTB, kShBits>(a, item, warp, lane, s_part);
     } else {
       const int r = item - n_shared;
       const int e = s_list.id[r / quads];
@@ -735,7 +736,7 @@ __device__ __forceinline__ void down_routed_tile(const DecodeDownArgs& a, int e,
   __syncthreads();
 }
 
-template <int NT>
+template <int NT, int kShBits>
 __device__ __forceinline__ void down_shared_tile(const DecodeDownArgs& a, int tile, int warp, int lane, float* s_part) {
   const int d = a.c.d, f = a.c.f, T = a.c.T;
   const int g = lane >> 2, t = lane & 3;
@@ -746,14 +747,14 @@ __device__ __forceinline__ void down_shared_tile(const DecodeDownArgs& a, int ti
   float acc[NT][4];
 #pragma unroll
   for (int n = 0; n < NT; ++n) acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.0f;
-  shared_rows<NT>(a.sh_down.w, a.sh_bits, drow, drow + 8, f, tok, kDownWarps, warp, lane, acc);
+  shared_rows<NT, kShBits>(a.sh_down.w, drow, drow + 8, f, tok, kDownWarps, warp, lane, acc);
 #pragma unroll
   for (int n = 0; n < NT; ++n)
 #pragma unroll
     for (int i = 0; i < 4; ++i) s_part[(warp * NT * 4 + n * 4 + i) * 32 + lane] = acc[n][i];
   __syncthreads();
-  const float sc_lo = a.sh_bits == 16 ? 1.0f : a.sh_down.scale[drow];
-  const float sc_hi = a.sh_bits == 16 ? 1.0f : a.sh_down.scale[drow + 8];
+  const float sc_lo = kShBits == 16 ? 1.0f : a.sh_down.scale[drow];
+  const float sc_hi = kShBits == 16 ? 1.0f : a.sh_down.scale[drow + 8];
   for (int n = warp; n < NT; n += kDownWarps) {
     float v[4];
 #pragma unroll
@@ -803,7 +804,7 @@ __device__ __forceinline__ void down_tile_done(const DecodeDownArgs& a, int tile
   __syncthreads();
 }
 
-template <int NTB>
+template <int NTB, int kShBits>
 __global__ void __launch_bounds__(kDownWarps * 32) decode_down_kernel(DecodeDownArgs a) {
   __shared__ ExpertList s_list;
   __shared__ int s_last;
@@ -825,7 +826,7 @@ __global__ void __launch_bounds__(kDownWarps * 32) decode_down_kernel(DecodeDown
       waited = true;
     }
     if (item < n_shared) {
-      down_shared_tile<NTB>(a, item, warp, lane, s_part);
+      down_shared_tile<NTB, kShBits>(a, item, warp, lane, s_part);
       down_tile_done(a, item, 1 + s_list.n, &s_last);
     } else {
       const int r = item - n_shared;
@@ -894,10 +895,20 @@ mote_status_t launch_decode_stream(const DecodeStreamArgs& p, int phase, cudaStr
     const int tiles = f / 8, quads = (tiles + kGuWarps - 1) / kGuWarps;
     const int max_items = tiles + std::min<int>(E, T * k) * quads;
     const int grid = std::min(max_items, sms * 12);
-    if (ntb == 1) MOTE_CUDA_OK(launch_pdl(decode_gateup_kernel<1>, dim3(grid), dim3(kGuWarps * 32), 0, stream, ga));
-    else if (ntb == 2) MOTE_CUDA_OK(launch_pdl(decode_gateup_kernel<2>, dim3(grid), dim3(kGuWarps * 32), 0, stream, ga));
-    else if (ntb == 4) MOTE_CUDA_OK(launch_pdl(decode_gateup_kernel<4>, dim3(grid), dim3(kGuWarps * 32), 0, stream, ga));
-    else MOTE_CUDA_OK(launch_pdl(decode_gateup_kernel<8>, dim3(grid), dim3(kGuWarps * 32), 0, stream, ga));
+#define MOTE_GU_LAUNCH(NTB_, BITS_) \
+  MOTE_CUDA_OK(launch_pdl(decode_gateup_kernel<NTB_, BITS_>, dim3(grid), dim3(kGuWarps * 32), 0, stream, ga))
+#define MOTE_GU_BITS(NTB_)                                 \
+  do {                                                     \
+    if (p.shared_bits == 8) MOTE_GU_LAUNCH(NTB_, 8);       \
+    else if (p.shared_bits == 4) MOTE_GU_LAUNCH(NTB_, 4);  \
+    else MOTE_GU_LAUNCH(NTB_, 16);                         \
+  } while (0)
+    if (ntb == 1) MOTE_GU_BITS(1);
+    else if (ntb == 2) MOTE_GU_BITS(2);
+    else if (ntb == 4) MOTE_GU_BITS(4);
+    else MOTE_GU_BITS(8);
+#undef MOTE_GU_BITS
+#undef MOTE_GU_LAUNCH
     ++g_launch_count;
     MOTE_LAUNCH_OK();
     return MOTE_OK;
@@ -915,13 +926,25 @@ mote_status_t launch_decode_stream(const DecodeStreamArgs& p, int phase, cudaStr
   const size_t smem = size_t(kDownWarps) * ntb * 4 * 32 * sizeof(float);
   static bool down_attr_set = false;
   if (!down_attr_set) {
-    MOTE_CUDA_OK(cudaFuncSetAttribute(decode_down_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 65536));
+    MOTE_CUDA_OK(cudaFuncSetAttribute(decode_down_kernel<8, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 65536));
+    MOTE_CUDA_OK(cudaFuncSetAttribute(decode_down_kernel<8, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 65536));
+    MOTE_CUDA_OK(cudaFuncSetAttribute(decode_down_kernel<8, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 65536));
     down_attr_set = true;
   }
-  if (ntb == 1) MOTE_CUDA_OK(launch_pdl(decode_down_kernel<1>, dim3(grid), dim3(kDownWarps * 32), smem, stream, da));
-  else if (ntb == 2) MOTE_CUDA_OK(launch_pdl(decode_down_kernel<2>, dim3(grid), dim3(kDownWarps * 32), smem, stream, da));
-  else if (ntb == 4) MOTE_CUDA_OK(launch_pdl(decode_down_kernel<4>, dim3(grid), dim3(kDownWarps * 32), smem, stream, da));
-  else MOTE_CUDA_OK(launch_pdl(decode_down_kernel<8>, dim3(grid), dim3(kDownWarps * 32), smem, stream, da));
+#define MOTE_DN_LAUNCH(NTB_, BITS_) \
+  MOTE_CUDA_OK(launch_pdl(decode_down_kernel<NTB_, BITS_>, dim3(grid), dim3(kDownWarps * 32), smem, stream, da))
+#define MOTE_DN_BITS(NTB_)                                 \
+  do {                                                     \
+    if (p.shared_bits == 8) MOTE_DN_LAUNCH(NTB_, 8);       \
+    else if (p.shared_bits == 4) MOTE_DN_LAUNCH(NTB_, 4);  \
+    else MOTE_DN_LAUNCH(NTB_, 16);                         \
+  } while (0)
+  if (ntb == 1) MOTE_DN_BITS(1);
+  else if (ntb == 2) MOTE_DN_BITS(2);
+  else if (ntb == 4) MOTE_DN_BITS(4);
+  else MOTE_DN_BITS(8);
+#undef MOTE_DN_BITS
+#undef MOTE_DN_LAUNCH
   ++g_launch_count;
   MOTE_LAUNCH_OK();
   return MOTE_OK;

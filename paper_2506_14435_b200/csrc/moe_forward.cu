@@ -311,22 +311,6 @@ extern "C" mote_status_t mote_moe_forward(const mote_layer_t* L, const void* x, 
 
   mote_status_t st;
   MOTE_CUDA_OK(cudaMemsetAsync(status, 0, 4, stream));
-  // prefill with an RTN-coded shared expert and room in the workspace: expand the codes to bf16 once
-  SharedMat xg = sh_gate, xu = sh_up, xd = sh_down;
-  int x_bits = sh_bits;
-  if (sh_rtn && tensor && T >= kExpandMinTokens && ws_bytes >= pl.total_expanded) {
-    char* e0 = base + pl.sh_codes_bf16;
-    const size_t mat = size_t(d) * f * 2;
-    ExpandArgs ea{};
-    for (int i = 0; i < 3; ++i) {
-      ea.codes[i] = static_cast<const uint4*>(i == 0 ? sh_gate.w : i == 1 ? sh_up.w : sh_down.w);
-      ea.out[i] = reinterpret_cast<uint4*>(e0 + i * mat);
-    }
-    st = launch_expand_codes(ea, int64_t(d) * f, sh_bits, stream);
-    if (st) return st;
-    xg.w = e0; xu.w = e0 + mat; xd.w = e0 + 2 * mat;
-    x_bits = MOTE_SHARED_BF16;                     // bf16 operands; the row scales still apply
-  }
   stage_mark(0, stream);
   // S1 router, S2 dispatch
   // block-wise dispatch: the tensor-core router (d % 32 == 0) leaves per-block expert counts, a small
@@ -385,6 +369,22 @@ extern "C" mote_status_t mote_moe_forward(const mote_layer_t* L, const void* x, 
   if (st) return st;
   stage_mark(6, stream);
   // S7 shared expert
+  // prefill with an RTN-coded shared expert and room in the workspace: expand the codes to bf16 once
+  SharedMat xg = sh_gate, xu = sh_up, xd = sh_down;
+  int x_bits = sh_bits;
+  if (sh_rtn && tensor && T >= kExpandMinTokens && ws_bytes >= pl.total_expanded) {
+    char* e0 = base + pl.sh_codes_bf16;
+    const size_t mat = size_t(d) * f * 2;
+    ExpandArgs ea{};
+    for (int i = 0; i < 3; ++i) {
+      ea.codes[i] = static_cast<const uint4*>(i == 0 ? sh_gate.w : i == 1 ? sh_up.w : sh_down.w);
+      ea.out[i] = reinterpret_cast<uint4*>(e0 + i * mat);
+    }
+    st = launch_expand_codes(ea, int64_t(d) * f, sh_bits, stream);
+    if (st) return st;
+    xg.w = e0; xu.w = e0 + mat; xd.w = e0 + 2 * mat;
+    x_bits = MOTE_SHARED_BF16;                     // bf16 operands; the row scales still apply
+  }
   st = tensor ? launch_shared_umma(x, xg, xu, x_bits, true, T, d, f, hs, tiles_shared, max_mtiles_shared,
                                    status, nullptr, stream, pdl)
               : launch_shared_gateup_simt(x, sh_gate, sh_up, sh_bits, T, d, f, hs, stream);

@@ -314,6 +314,58 @@ mote_status_t launch_route_topk(const void* x, int64_t T, int d, const float* Wr
 
 }  // namespace mote
 
+namespace mote {
+
+// Per-expert factors of the load-balancing loss (Eq. 12): one CTA per expert walks the batch in a
+// fixed order (thread-strided partial sums, then a fixed tree), so the sums are reproducible.
+__global__ void __launch_bounds__(256) route_stats_kernel(const float* __restrict__ logits,
+                                                          const int32_t* __restrict__ idx, int64_t T, int E, int k,
+                                                          int32_t* __restrict__ tokens_per_expert,
+                                                          float* __restrict__ prob_sum) {
+  __shared__ float s_p[8];
+  __shared__ int s_c[8];
+  const int e = blockIdx.x;
+  float p = 0.0f;
+  int c = 0;
+  for (int64_t t = threadIdx.x; t < T; t += blockDim.x) {
+    const float* l = logits + t * E;
+    float m = l[0];
+    for (int j = 1; j < E; ++j) m = fmaxf(m, l[j]);
+    float den = 0.0f;
+    for (int j = 0; j < E; ++j) den += expf(l[j] - m);
+    p += expf(l[e] - m) / den;
+    for (int j = 0; j < k; ++j) c += (idx[t * k + j] == e) ? 1 : 0;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    p += __shfl_xor_sync(0xffffffffu, p, o);
+    c += __shfl_xor_sync(0xffffffffu, c, o);
+  }
+  if ((threadIdx.x & 31) == 0) { s_p[threadIdx.x >> 5] = p; s_c[threadIdx.x >> 5] = c; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float ps = 0.0f;
+    int cs = 0;
+    for (int w = 0; w < 8; ++w) { ps += s_p[w]; cs += s_c[w]; }
+    prob_sum[e] = ps;
+    tokens_per_expert[e] = cs;
+  }
+}
+
+}  // namespace mote
+
+extern "C" mote_status_t mote_route_stats(const float* logits, const int32_t* topk_idx, int64_t T, int E, int k,
+                                          int32_t* tokens_per_expert, float* prob_sum, void* stream) {
+  using namespace mote;
+  if (T < 0 || E < 1 || E > MOTE_MAX_EXPERTS || k < 1 || k > E || k > MOTE_MAX_TOPK) return MOTE_ERR_SHAPE;
+  if (!tokens_per_expert || !prob_sum) return MOTE_ERR_NULL;
+  if (T > 0 && (!logits || !topk_idx)) return MOTE_ERR_NULL;
+  route_stats_kernel<<<E, 256, 0, static_cast<cudaStream_t>(stream)>>>(logits, topk_idx, T, E, k, tokens_per_expert,
+                                                                       prob_sum);
+  MOTE_LAUNCH_OK();
+  return MOTE_OK;
+}
+
 extern "C" mote_status_t mote_route_topk(const void* x_bf16, int64_t T, int64_t d, const float* Wr,
                                          const float* bias, int E, int k, int norm_topk, int32_t* topk_idx,
                                          float* topk_w, float* logits, void* stream) {

@@ -96,3 +96,7 @@ def test_host_side_argument_errors(mote):
     assert lib.mote_rtn_quant(fake, 1, 4, 24, 8, fake, fake, NULL) == 2
     assert lib.mote_rtn_quant(fake, 1, 4, 16, 2, fake, fake, NULL) == 2
     assert lib.mote_rtn_quant(odd, 1, 4, 16, 4, fake, fake, NULL) == 3
+    # route_stats
+    assert lib.mote_route_stats(fake, fake, 4, 65, 2, fake, fake, NULL) == 2
+    assert lib.mote_route_stats(fake, fake, 4, 4, 2, NULL, fake, NULL) == 1
+    assert lib.mote_route_stats(NULL, fake, 4, 4, 2, fake, fake, NULL) == 1

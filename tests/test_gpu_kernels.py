@@ -180,3 +180,25 @@ def test_rtn_quant_ties_and_errors(mote, bits):
     with pytest.raises(mote.MoteError) as ei:
         mote.mote_rtn_quant(torch.zeros((4, 32), device="cuda"), 3)
     assert ei.value.status == 2
+
+
+@pytest.mark.parametrize("T,d,E,k,bias", [(1, 64, 4, 1, False), (300, 256, 8, 2, True), (4096, 896, 4, 2, False),
+                                          (777, 128, 64, 8, True)])
+def test_route_stats(mote, T, d, E, k, bias):
+    # Eq. 12: tokens per expert exactly, summed routing probabilities to fp32 accuracy
+    x = O.f32_to_bf16_rn(_randn((T, d), 60 + T, 1.0).astype(np.float32))
+    Wr = O.bf16_to_f32(O.f32_to_bf16_rn(_randn((E, d), 61 + T, 0.05).astype(np.float32)))
+    b = _randn((E,), 62 + T, 0.5).astype(np.float32) if bias else None
+    idx, w, logits = mote.mote_route_topk(bf16_tensor(x), torch.from_numpy(Wr).cuda(),
+                                          None if b is None else torch.from_numpy(b).cuda(), k, want_logits=True)
+    cnt, ps = mote.mote_route_stats(logits, idx)
+    t_ref, s_ref = O.load_balance_stats(logits.cpu().numpy(), idx.cpu().numpy(), E)
+    assert np.array_equal(cnt.cpu().numpy(), t_ref)
+    assert np.allclose(ps.cpu().numpy(), s_ref, rtol=2e-5, atol=1e-6)
+    assert cnt.sum().item() == T * k and abs(ps.sum().item() - T) <= 1e-4 * T
+    # against the oracle's own router (fp64 logits): same counts away from near ties
+    r = O.router(x, Wr, b, k, 1)
+    if not r["near_tie"].any():
+        t2, s2 = O.load_balance_stats(r["logits"], r["idx"], E)
+        assert np.array_equal(cnt.cpu().numpy(), t2)
+        assert np.allclose(ps.cpu().numpy(), s2, rtol=1e-4, atol=1e-5)
