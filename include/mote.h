@@ -51,7 +51,8 @@ enum { MOTE_SHARED_BF16 = 16, MOTE_SHARED_INT8 = 8, MOTE_SHARED_INT4 = 4 };
  * the tests to check every path against the oracle).
  *   STREAM  decode, T <= 64 with d % 64 == 0, f % 64 == 0, d <= 16384, T*k <= 512: the weights are
  *           streamed once from HBM through registers into warp-level MMAs
- *   TENSOR  d % 128 == 0 and f % 128 == 0: tcgen05 GEMMs (int8 x 2-bit routed, bf16 shared)
+ *   TENSOR  d % 128 == 0 and f % 128 == 0: tcgen05 GEMMs (int8 x 2-bit routed, bf16 shared; an
+ *           RTN-coded shared expert is expanded to bf16 on the way, see mote_layer_workspace_bytes)
  *   SIMT    any d, f that are multiples of 16: CUDA-core GEMMs
  * AUTO takes the first of these whose conditions hold. */
 enum { MOTE_PATH_AUTO = 0, MOTE_PATH_SIMT = 1, MOTE_PATH_TENSOR = 2, MOTE_PATH_STREAM = 3 };
@@ -298,8 +299,9 @@ mote_status_t mote_stack_forward(const mote_layer_t* layers_host, int n_layers, 
  *   5 down ternary GEMM (Eq. 5)   6 shared gate/up   7 shared down (Eq. 2)   8 combine (Eq. 2, 4)
  * A stage that a path folds into its neighbour reports 0: the tensor path does the combine in the
  * shared-down epilogue (stage 7); the decode path reports its prologue (Q_a(x), router, dispatch)
- * as stage 0 and its two streaming kernels, which cover the routed AND the shared expert, as
- * stages 3 and 5.  Stages run back to back on one
+ * as stage 0 and its two streaming kernels, which cover the routed AND the shared expert (and, in
+ * the second one, the combine), as stages 3 and 5.  An RTN prefill's code expansion counts
+ * into stage 6.  Stages run back to back on one
  * stream here even if mote_moe_forward overlaps some of them. */
 enum { MOTE_N_STAGES = 9 };
 mote_status_t mote_moe_forward_profile(const mote_layer_t* L, const void* x_bf16,
