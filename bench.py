@@ -191,7 +191,12 @@ def run_ours(args):
     out = torch.empty_like(x)
     flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
     stream = torch.cuda.current_stream()
-    stream_path = wl.T <= 64 and wl.d % 64 == 0 and wl.f % 64 == 0
+    if args.path != "auto":                             # force one implementation (default: the library picks)
+        for l in layers:
+            l.path = {"simt": mote.PATH_SIMT, "tensor": mote.PATH_TENSOR, "stream": mote.PATH_STREAM}[args.path]
+        if is_stack:
+            stack = mote.MoteStack(layers)
+    stream_path = (wl.T <= 64 and wl.d % 64 == 0 and wl.f % 64 == 0) if args.path == "auto" else args.path == "stream"
 
     def step_device():
         if is_stack:
@@ -335,7 +340,7 @@ def run_ours(args):
             "" if args.shared_bits == 16 else f" (weights RTN int{args.shared_bits}, weight-only)"), "data": "synthetic",
         "config": {"workload": wl.name, "d": wl.d, "f": wl.f, "E": wl.E, "k": wl.k, "T_per_gpu": wl.T,
                    "layers": len(layers), "experts_touched_per_layer": experts_touched,
-                   "shared_bits": args.shared_bits,
+                   "shared_bits": args.shared_bits, "path": args.path,
                    "launch": "CUDA graph replay of the step" if args.graph else "direct launches",
                    "pre_norm": "rms, eps 1e-6, unit gain" if is_stack else "none (the caller's)",
                    "l2": "flushed between timed iterations (512 MiB write)", "parallelism": f"replicas x{world}"},
@@ -425,6 +430,8 @@ def main():
     ap.add_argument("--layers", type=int, default=None, help="layers of a stacked workload (c5-T: default 36)")
     ap.add_argument("--shared-bits", type=int, default=16, choices=[16, 8, 4],
                     help="storage of the shared expert: bf16, or RTN INT8 / INT4 codes (Section 4.3)")
+    ap.add_argument("--path", default="auto", choices=["auto", "simt", "tensor", "stream"],
+                    help="implementation of the layer (auto: the library's own choice per shape)")
     ap.add_argument("--graph", action="store_true",
                     help="time the step as a CUDA graph replay (captured once from the same C-ABI call)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])

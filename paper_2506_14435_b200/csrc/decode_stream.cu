@@ -313,12 +313,21 @@ __device__ __forceinline__ void ternary_rows_steps(const uint8_t* __restrict__ r
             fa[j] = (wa[w] >> (2 * j)) & 0x03030303u;
             fb[j] = (wb[w] >> (2 * j)) & 0x03030303u;
           }
+          // the token fragments of up to four column tiles first (independent loads), then their MMAs
+          constexpr int kG = NT < 4 ? NT : 4;
 #pragma unroll
-          for (int n = 0; n < NT; ++n) {
-            uint4 q = make_uint4(0u, 0u, 0u, 0u);
-            if (tok[n] && q_ok) q = *reinterpret_cast<const uint4*>(tok[n] + q_off + w * 16);
-            mma_u8s8(acc[n], fa[0], fb[0], fa[1], fb[1], q.x, q.y);
-            mma_u8s8(acc[n], fa[2], fb[2], fa[3], fb[3], q.z, q.w);
+          for (int n0 = 0; n0 < NT; n0 += kG) {
+            uint4 q[kG];
+#pragma unroll
+            for (int n = 0; n < kG; ++n) {
+              q[n] = make_uint4(0u, 0u, 0u, 0u);
+              if (tok[n0 + n] && q_ok) q[n] = *reinterpret_cast<const uint4*>(tok[n0 + n] + q_off + w * 16);
+            }
+#pragma unroll
+            for (int n = 0; n < kG; ++n) {
+              mma_u8s8(acc[n0 + n], fa[0], fb[0], fa[1], fb[1], q[n].x, q[n].y);
+              mma_u8s8(acc[n0 + n], fa[2], fb[2], fa[3], fb[3], q[n].z, q[n].w);
+            }
           }
         }
       }
@@ -351,12 +360,20 @@ __device__ __forceinline__ void bf16_rows_steps(const uint16_t* __restrict__ row
           qa[i] = ldg_stream16(row_a + (s + kBf16Ahead) * 32 + t * 8);
           qb[i] = ldg_stream16(row_b + (s + kBf16Ahead) * 32 + t * 8);
         }
+        constexpr int kG = NT < 4 ? NT : 4;
 #pragma unroll
-        for (int n = 0; n < NT; ++n) {
-          uint4 q = kZero;
-          if (tok[n]) q = *reinterpret_cast<const uint4*>(tok[n] + s * 32 + t * 8);
-          mma_bf16(acc[n], ca.x, cb.x, ca.y, cb.y, q.x, q.y);
-          mma_bf16(acc[n], ca.z, cb.z, ca.w, cb.w, q.z, q.w);
+        for (int n0 = 0; n0 < NT; n0 += kG) {
+          uint4 q[kG];
+#pragma unroll
+          for (int n = 0; n < kG; ++n) {
+            q[n] = kZero;
+            if (tok[n0 + n]) q[n] = *reinterpret_cast<const uint4*>(tok[n0 + n] + s * 32 + t * 8);
+          }
+#pragma unroll
+          for (int n = 0; n < kG; ++n) {
+            mma_bf16(acc[n0 + n], ca.x, cb.x, ca.y, cb.y, q[n].x, q[n].y);
+            mma_bf16(acc[n0 + n], ca.z, cb.z, ca.w, cb.w, q[n].z, q[n].w);
+          }
         }
       }
     }
@@ -404,22 +421,36 @@ __device__ __forceinline__ void rtn_rows_steps(const uint8_t* __restrict__ row_a
             uint32_t a01, a23, b01, b23;
             s8x4_to_bf16x2(wa[w], a01, a23);
             s8x4_to_bf16x2(wb[w], b01, b23);
+            constexpr int kG = NT < 4 ? NT : 4;
 #pragma unroll
-            for (int n = 0; n < NT; ++n) {
-              uint2 q = make_uint2(0u, 0u);
-              if (tok[n] && q_ok) q = *reinterpret_cast<const uint2*>(tok[n] + e0 + 4 * w);
-              mma_bf16(acc[n], a01, b01, a23, b23, q.x, q.y);
+            for (int n0 = 0; n0 < NT; n0 += kG) {
+              uint2 q[kG];
+#pragma unroll
+              for (int n = 0; n < kG; ++n) {
+                q[n] = make_uint2(0u, 0u);
+                if (tok[n0 + n] && q_ok) q[n] = *reinterpret_cast<const uint2*>(tok[n0 + n] + e0 + 4 * w);
+              }
+#pragma unroll
+              for (int n = 0; n < kG; ++n) mma_bf16(acc[n0 + n], a01, b01, a23, b23, q[n].x, q[n].y);
             }
           } else {
             uint32_t ea[4], eb[4];
             u4x8_to_bf16x2(wa[w], ea);
             u4x8_to_bf16x2(wb[w], eb);
+            constexpr int kG = NT < 4 ? NT : 4;
 #pragma unroll
-            for (int n = 0; n < NT; ++n) {
-              uint4 q = make_uint4(0u, 0u, 0u, 0u);
-              if (tok[n] && q_ok) q = *reinterpret_cast<const uint4*>(tok[n] + e0 + 8 * w);
-              mma_bf16(acc[n], ea[0], eb[0], ea[1], eb[1], q.x, q.y);
-              mma_bf16(acc[n], ea[2], eb[2], ea[3], eb[3], q.z, q.w);
+            for (int n0 = 0; n0 < NT; n0 += kG) {
+              uint4 q[kG];
+#pragma unroll
+              for (int n = 0; n < kG; ++n) {
+                q[n] = make_uint4(0u, 0u, 0u, 0u);
+                if (tok[n0 + n] && q_ok) q[n] = *reinterpret_cast<const uint4*>(tok[n0 + n] + e0 + 8 * w);
+              }
+#pragma unroll
+              for (int n = 0; n < kG; ++n) {
+                mma_bf16(acc[n0 + n], ea[0], eb[0], ea[1], eb[1], q[n].x, q[n].y);
+                mma_bf16(acc[n0 + n], ea[2], eb[2], ea[3], eb[3], q[n].z, q[n].w);
+              }
             }
           }
         }
