@@ -49,6 +49,9 @@ def test_c1_full_parity(mote, path):
     (128, 256, 8, 2, 77, dict(bias="zipf"), TENSOR),
     (128, 384, 4, 1, 130, dict(norm_topk=0), TENSOR),     # down projection with 128-wide tiles
     (384, 640, 3, 3, 515, {}, TENSOR),                    # k = E, several row tiles per expert
+    (128, 256, 64, 8, 200, {}, TENSOR),                   # many experts, k = 8: 128 pairs per router block
+    (256, 128, 16, 4, 1000, dict(bias="normal"), TENSOR), # more row tiles than experts, uneven loads
+    (128, 256, 64, 8, 70, {}, SIMT),
     (64, 128, 3, 3, 5, {}, STREAM),                       # k = E, one short reduction step
     (128, 192, 2, 1, 1, {}, STREAM),                      # one token
     (896, 4864, 4, 2, 17, dict(outlier_frac=0.01), STREAM),   # d/4 = 224 bytes: a ragged last step
