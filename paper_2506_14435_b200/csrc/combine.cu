@@ -1,5 +1,6 @@
 // Gate-weighted combine and un-permute (Eq. 2, Eq. 4), gather form (no atomics, deterministic):
 //   out[t,:] = bf16( [residual[t,:] +] s[t,:] + sum_{j<k} w[t,j] * y[perm[t*k+j], :] )
+// (s may arrive as the partial sums of a K-split down projection, added here in ascending order)
 // fp32 arithmetic, slots added in ascending j, one bf16 rounding at the end.
 // HBM-bound: per output element 4 B (s) + 4k B (y) [+ 2 B residual] read, 2 B written.
 #include "mote_common.cuh"
@@ -10,7 +11,7 @@ namespace mote {
 __global__ void __launch_bounds__(256) combine_kernel(const float* __restrict__ s, const float* __restrict__ y,
                                                       const float* __restrict__ w, const int32_t* __restrict__ perm,
                                                       const uint16_t* residual, int64_t T, int d, int k,
-                                                      uint16_t* out) {
+                                                      uint16_t* out, int n_partials) {
   const int vec_per_row = d / 8;
   const int64_t total = T * vec_per_row;
   pdl_wait();                            // no-op unless launched as a programmatic dependent
@@ -24,6 +25,12 @@ __global__ void __launch_bounds__(256) combine_kernel(const float* __restrict__ 
       const float4 a = sp[0], b = sp[1];
       acc[0] = a.x; acc[1] = a.y; acc[2] = a.z; acc[3] = a.w;
       acc[4] = b.x; acc[5] = b.y; acc[6] = b.z; acc[7] = b.w;
+    }
+    for (int p = 1; p < n_partials; ++p) {           // partial sums of a K-split projection, in order
+      const float4* sp = reinterpret_cast<const float4*>(s + (int64_t(p) * T + t) * d + v * 8);
+      const float4 a = sp[0], b = sp[1];
+      acc[0] += a.x; acc[1] += a.y; acc[2] += a.z; acc[3] += a.w;
+      acc[4] += b.x; acc[5] += b.y; acc[6] += b.z; acc[7] += b.w;
     }
     for (int j = 0; j < k; ++j) {
       const float wj = w[t * k + j];
@@ -50,16 +57,17 @@ __global__ void __launch_bounds__(256) combine_kernel(const float* __restrict__ 
 
 mote_status_t launch_combine(const float* s, const float* y, const float* w, const int32_t* perm,
                              const void* residual, int64_t T, int d, int k, void* out_bf16, cudaStream_t stream,
-                             bool pdl) {
+                             bool pdl, int n_partials) {
   if (T == 0) return MOTE_OK;
   const int64_t total = T * (d / 8);
   const unsigned blocks = (unsigned)std::min<int64_t>((total + 255) / 256, 148 * 16);
   if (pdl)
     MOTE_CUDA_OK(launch_pdl(combine_kernel, dim3(blocks), dim3(256), 0, stream, s, y, w, perm,
-                            static_cast<const uint16_t*>(residual), T, d, k, static_cast<uint16_t*>(out_bf16)));
+                            static_cast<const uint16_t*>(residual), T, d, k, static_cast<uint16_t*>(out_bf16),
+                            n_partials));
   else
     combine_kernel<<<blocks, 256, 0, stream>>>(s, y, w, perm, static_cast<const uint16_t*>(residual), T, d, k,
-                                               static_cast<uint16_t*>(out_bf16));
+                                               static_cast<uint16_t*>(out_bf16), n_partials);
   ++g_launch_count;
   MOTE_LAUNCH_OK();
   return MOTE_OK;

@@ -61,7 +61,8 @@ static Plan make_plan(int d, int f, int E, int k, int64_t T) {
   p.rowsum_h = take(P * 4);
   p.y = take(P * size_t(d) * 4);
   p.hs = take(size_t(T) * f * 2);
-  p.s = take(size_t(T) * d * 4);
+  // room for the partial outputs of a K-split shared down projection (short prefills)
+  p.s = take(size_t(std::max<int64_t>(T, std::min<int64_t>(kMaxPartialRows, 16 * T))) * d * 4);
   p.tiles_routed = take((1 + P / 128 + E) * 16);
   p.tiles_shared = take((1 + (size_t(T) + 127) / 128) * 16);
   const size_t n_blk = (size_t(T) + kRouteBlockTokens - 1) / kRouteBlockTokens;
@@ -136,6 +137,15 @@ __global__ void copy_q_rows_kernel(const int8_t* __restrict__ src, int8_t* __res
     }
     reinterpret_cast<uint4*>(dst)[r * n_units + u] = v;
   }
+}
+
+// dst[i] = sum_p src[p * n + i], p ascending (the partial outputs of a K-split projection; tap only)
+__global__ void sum_partials_kernel(const float* __restrict__ src, int n_partials, int64_t n, float* __restrict__ dst) {
+  const int64_t i = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  float acc = src[i];
+  for (int p = 1; p < n_partials; ++p) acc += src[int64_t(p) * n + i];
+  dst[i] = acc;
 }
 
 __global__ void gather_f32_kernel(const float* __restrict__ src, float* __restrict__ dst, int64_t n,
@@ -390,7 +400,16 @@ extern "C" mote_status_t mote_moe_forward(const mote_layer_t* L, const void* x, 
               : launch_shared_gateup_simt(x, sh_gate, sh_up, sh_bits, T, d, f, hs, stream);
   if (st) return st;
   stage_mark(7, stream);
-  if (tensor) {
+  const int k_splits = tensor ? shared_down_k_splits(T, d, f) : 1;
+  if (tensor && k_splits > 1) {
+    // few row tiles: the shared down projection is cut along K, its partial outputs are added by the combine
+    st = launch_shared_umma(hs, xd, SharedMat{nullptr, nullptr}, x_bits, false, T, f, d, s, tiles_shared,
+                            max_mtiles_shared, status, nullptr, stream, pdl, k_splits);
+    if (st) return st;
+    stage_mark(8, stream);
+    st = launch_combine(s, y, topk_w, perm, residual, T, d, k, out, stream, pdl, k_splits);
+    if (st) return st;
+  } else if (tensor) {
     // shared down projection with S8 (combine, residual, bf16 rounding) in its epilogue; the fp32
     // shared output is written only when a tap asks for it
     CombineArgs cb{y, topk_w, perm, residual, out, k};
@@ -416,8 +435,14 @@ extern "C" mote_status_t mote_moe_forward(const mote_layer_t* L, const void* x, 
     bool ok = d2d(taps->topk_idx, topk_idx, P * 4) && d2d(taps->topk_w, topk_w, P * 4) &&
               d2d(taps->offsets, offsets, size_t(E + 1) * 4) && d2d(taps->perm, perm, P * 4) &&
               d2d(taps->h_bf16, h, size_t(P) * f * 2) && d2d(taps->beta_h, beta_h, P * 4) &&
-              d2d(taps->y, y, size_t(P) * d * 4) && d2d(taps->shared_out, s, size_t(T) * d * 4);
+              d2d(taps->y, y, size_t(P) * d * 4) &&
+              (k_splits > 1 || d2d(taps->shared_out, s, size_t(T) * d * 4));
     if (!ok) return MOTE_ERR_CUDA;
+    if (k_splits > 1 && taps->shared_out) {
+      const int64_t n = T * d;
+      sum_partials_kernel<<<(unsigned)((n + 255) / 256), 256, 0, stream>>>(s, k_splits, n, taps->shared_out);
+      MOTE_LAUNCH_OK();
+    }
     if (taps->qx) {
       copy_q_rows_kernel<<<148 * 4, 256, 0, stream>>>(qx, taps->qx, T, d / 16, perm, k, interleave);
       MOTE_LAUNCH_OK();

@@ -91,9 +91,14 @@ struct SharedMat { const void* w; const float* scale; };
 struct CombineArgs {
   const float* y; const float* w; const int32_t* perm; const void* residual; void* out; int k;
 };
+// k_splits > 1 (down projection only, no comb): `out` receives k_splits partial outputs of T x N
+// floats each, to be added in ascending order (see shared_down_k_splits).
 mote_status_t launch_shared_umma(const void* act, const SharedMat& w0, const SharedMat& w1, int bits, bool gateup,
                                  int64_t T, int K, int N, void* out, const int4* tiles, int max_mtiles,
-                                 uint32_t* status, const CombineArgs* comb, cudaStream_t stream, bool pdl = false);
+                                 uint32_t* status, const CombineArgs* comb, cudaStream_t stream, bool pdl = false,
+                                 int k_splits = 1);
+constexpr int64_t kMaxPartialRows = 4096;
+int shared_down_k_splits(int64_t T, int N, int K);
 
 // CUDA-core GEMMs of the shared expert.
 mote_status_t launch_shared_gateup_simt(const void* x, const SharedMat& Wg, const SharedMat& Wu, int bits, int64_t T,
@@ -126,8 +131,9 @@ mote_status_t launch_decode_stream(const DecodeStreamArgs& a, int phase, cudaStr
 mote_status_t launch_rms_norm(const void* x, int64_t T, int d, float eps, void* y, cudaStream_t stream);
 
 // out = [residual +] s + sum_j w_j * y[perm[t*k+j]]
+// s may hold n_partials partial outputs of T x d floats each; they are added in ascending order.
 mote_status_t launch_combine(const float* s, const float* y, const float* w, const int32_t* perm,
                              const void* residual, int64_t T, int d, int k, void* out_bf16,
-                             cudaStream_t stream, bool pdl = false);
+                             cudaStream_t stream, bool pdl = false, int n_partials = 1);
 
 }  // namespace mote

@@ -57,6 +57,8 @@ struct UmmaArgs {
   const int4* tiles;        // [0] = {n_mtiles,0,0,0}; [1+i] = {expert, row0, rows, 0}
   int n_ntiles;             // tiles along the output columns
   int k_steps;              // pipeline stages along K (128 bytes of the token operand each)
+  int k_splits;             // down projections: items per output tile, each over 1/k_splits of K (>= 1)
+  int64_t split_stride;     // elements between the partial outputs of consecutive splits
   int bn;                   // weight rows per tile (UMMA N)
   int n_out;                // output row length (f for gate/up, d for down)
   int b_rows_per_expert;    // rows of the weight tensor map per expert (0: shared expert)
@@ -111,12 +113,22 @@ struct ModeTraits {
 //            (T x d) stays in L2 across column tiles;
 //   down:    column tile fastest -- concurrent items share the token operand (P x f, larger than
 //            L2 for long prefills), which is then read from HBM once instead of once per column tile.
+// A down projection with few row tiles may split K over k_splits items per output tile (each
+// writes its partial sums; the caller adds them in a fixed order): item = (row tile, split, column tile).
 template <bool kGateUp>
 __device__ __forceinline__ void decode_item(const UmmaArgs& a, int item, int n_mtiles, int4& tile, int& n_tile) {
   int m_tile;
   if (kGateUp) { m_tile = item % n_mtiles; n_tile = item / n_mtiles; }
-  else { m_tile = item / a.n_ntiles; n_tile = item % a.n_ntiles; }
+  else { m_tile = item / (a.n_ntiles * a.k_splits); n_tile = item % a.n_ntiles; }
   tile = a.tiles[1 + m_tile];
+}
+// pipeline steps [kb, ke) of an item, and which split it is
+__device__ __forceinline__ int item_k_range(const UmmaArgs& a, int item, int& kb, int& ke) {
+  if (a.k_splits <= 1) { kb = 0; ke = a.k_steps; return 0; }
+  const int split = (item / a.n_ntiles) % a.k_splits;
+  kb = split * a.k_steps / a.k_splits;
+  ke = (split + 1) * a.k_steps / a.k_splits;
+  return split;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -168,7 +180,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
   const uint32_t tmem_base = bars->tmem_base;
   pdl_wait();                              // set-up above overlaps the tail of the kernel before this one
   const int n_mtiles = a.tiles[0].x;
-  const int n_items = n_mtiles * a.n_ntiles;
+  const int n_items = n_mtiles * a.n_ntiles * a.k_splits;
 
   if (warp == 0) {
     // ---------------------------------------------------------------- token-operand producer
@@ -179,7 +191,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
         int4 tile; int n_tile;
         decode_item<TR::kGateUp>(a, item, n_mtiles, tile, n_tile);
         const int b_row = (a.b_rows_per_expert ? tile.x * a.b_rows_per_expert : 0) + n_tile * (TR::kGateUp ? a.bn / 2 : a.bn);
-        for (int ks = 0; ks < a.k_steps; ++ks) {
+        int kb, ke;
+        item_k_range(a, item, kb, ke);
+        for (int ks = kb; ks < ke; ++ks) {
           if (!(ok = mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1, abort_flag))) break;
           const uint32_t bar = smem_u32(&bars->full_a[stage]);
           if (TR::kTernary) {
@@ -213,7 +227,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
         int4 tile; int n_tile;
         decode_item<TR::kGateUp>(a, item, n_mtiles, tile, n_tile);
         const int b_row = tile.x * a.b_rows_per_expert + n_tile * (TR::kGateUp ? a.bn / 2 : a.bn);
-        for (int ks = 0; ks < a.k_steps; ++ks) {
+        int kb, ke;
+        item_k_range(a, item, kb, ke);
+        for (int ks = kb; ks < ke; ++ks) {
           if (!(ok = mbar_wait(smem_u32(&bars->empty_p[stage]), phase ^ 1, abort_flag))) break;
           const uint32_t bar = smem_u32(&bars->full_p[stage]);
           mbar_expect_tx(bar, a.bn * kRB);
@@ -243,7 +259,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
         if (!(ok = mbar_wait(smem_u32(&bars->tmem_empty[buf]), (use & 1) ^ 1, abort_flag))) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * 256;
-        for (int ks = 0; ks < a.k_steps; ++ks) {
+        int kb, ke;
+        item_k_range(a, item, kb, ke);
+        for (int ks = kb; ks < ke; ++ks) {
           if (!(ok = mbar_wait(smem_u32(&bars->full_a[stage]), phase, abort_flag))) break;
           if (TR::kUnpack)
             if (!(ok = mbar_wait(smem_u32(&bars->full_u[stage]), phase, abort_flag))) break;
@@ -252,7 +270,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
           const uint64_t db = smem_desc_sw128(sB + stage * kStageB);
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
-            const uint32_t acc = (ks > 0 || j > 0) ? 1u : 0u;
+            const uint32_t acc = (ks > kb || j > 0) ? 1u : 0u;
             if (TR::kTernary) mma_i8(d_tmem, da + 2 * j, db + 2 * j, idesc, acc);
             else mma_f16(d_tmem, da + 2 * j, db + 2 * j, idesc, acc);
           }
@@ -273,7 +291,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
       bool ok = true;
       const int n_chunks = a.bn * (TR::kCodeRowBytes / 16);   // chunks of 16 code bytes, spread over 128 threads
       for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x) {
-        for (int ks = 0; ks < a.k_steps; ++ks, ++step) {
+        int kb, ke;
+        item_k_range(a, item, kb, ke);
+        for (int ks = kb; ks < ke; ++ks, ++step) {
           if ((step & 1u) == (uint32_t)group) {
             ok = mbar_wait(smem_u32(&bars->full_p[pstage]), pphase, abort_flag) &&
                  mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1, abort_flag);
@@ -347,6 +367,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
     for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x, ++local) {
       int4 tile; int n_tile;
       decode_item<TR::kGateUp>(a, item, n_mtiles, tile, n_tile);
+      int kb_, ke_;
+      const int split = item_k_range(a, item, kb_, ke_);
       const int buf = local & 1;
       const uint32_t use = (uint32_t)(local >> 1);
       ok = mbar_wait(smem_u32(&bars->tmem_full[buf]), use & 1, abort_flag);
@@ -495,7 +517,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
               }
             }
             if (a.out) {
-              float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(a.out) + row * a.n_out + col0 + c);
+              float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(a.out) + split * a.split_stride +
+                                                      row * a.n_out + col0 + c);
 #pragma unroll
               for (int v = 0; v < 4; ++v) dst[v] = make_float4(o[4 * v], o[4 * v + 1], o[4 * v + 2], o[4 * v + 3]);
             }
@@ -641,6 +664,7 @@ mote_status_t launch_ternary_umma(const TernaryGemmArgs& g, bool gateup, const i
   a.tiles = tiles;
   a.n_ntiles = gateup ? g.N / 128 : g.N / bn;
   a.k_steps = g.K / 128;
+  a.k_splits = 1;
   a.bn = bn;
   a.n_out = g.N;
   a.b_rows_per_expert = g.N;
@@ -654,10 +678,30 @@ mote_status_t launch_ternary_umma(const TernaryGemmArgs& g, bool gateup, const i
                 : launch_umma<MODE_T_DOWN>(ta, tb0, tb1, a, max_items, stream, pdl);
 }
 
+// K splits of the shared down projection: with few row tiles its T x N output has too few tiles to
+// occupy the SMs (one row tile of c3: 6 tiles for 27 MB of weights), so each tile's K range is cut
+// into up to 16 items whose partial sums the caller adds.  At most 4096 partial rows in all.
+int shared_down_k_splits(int64_t T, int N, int K) {
+  static int sms = 0;
+  if (sms == 0) {
+    int dev = 0, v = 148;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev);
+    sms = v;
+  }
+  const int64_t n_tiles = ((T + 127) / 128) * (N / pick_bn(N));
+  if (n_tiles * 2 > sms) return 1;
+  int64_t splits = std::min<int64_t>(16, sms / n_tiles);
+  splits = std::min<int64_t>(splits, (K / 64) / 4);
+  splits = std::min<int64_t>(splits, kMaxPartialRows / T);
+  return (int)std::max<int64_t>(splits, 1);
+}
+
 mote_status_t launch_shared_umma(const void* act, const SharedMat& w0, const SharedMat& w1, int bits, bool gateup,
                                  int64_t T, int K, int N, void* out, const int4* tiles, int max_mtiles,
-                                 uint32_t* status, const CombineArgs* comb, cudaStream_t stream, bool pdl) {
+                                 uint32_t* status, const CombineArgs* comb, cudaStream_t stream, bool pdl,
+                                 int k_splits) {
   if (T == 0) return MOTE_OK;
+  if (k_splits > 1 && (gateup || comb || !out)) return MOTE_ERR_SHAPE;
   CUtensorMap ta, tb0, tb1;
   const int bn = gateup ? 256 : pick_bn(N);
   const uint32_t rows1 = (gateup || bn <= 128) ? 128 : bn - 128;
@@ -685,6 +729,8 @@ mote_status_t launch_shared_umma(const void* act, const SharedMat& w0, const Sha
   a.tiles = tiles;
   a.n_ntiles = gateup ? N / 128 : N / bn;
   a.k_steps = K / 64;
+  a.k_splits = std::max(k_splits, 1);
+  a.split_stride = T * N;
   a.bn = bn;
   a.n_out = N;
   a.b_rows_per_expert = 0;
@@ -696,7 +742,7 @@ mote_status_t launch_shared_umma(const void* act, const SharedMat& w0, const Sha
     a.comb_res = static_cast<const uint16_t*>(comb->residual); a.comb_out = static_cast<uint16_t*>(comb->out);
     a.comb_k = comb->k;
   }
-  const int max_items = max_mtiles * a.n_ntiles;
+  const int max_items = max_mtiles * a.n_ntiles * a.k_splits;
   if (bits == 8)
     return gateup ? launch_umma<MODE_Q8_GATEUP>(ta, tb0, tb1, a, max_items, stream, pdl)
                   : launch_umma<MODE_Q8_DOWN>(ta, tb0, tb1, a, max_items, stream, pdl);
