@@ -197,7 +197,9 @@ def run_ours(args):
             l.path = {"simt": mote.PATH_SIMT, "tensor": mote.PATH_TENSOR, "stream": mote.PATH_STREAM}[args.path]
         if is_stack:
             stack = mote.MoteStack(layers)
-    stream_path = (wl.T <= 64 and wl.d % 64 == 0 and wl.f % 64 == 0) if args.path == "auto" else args.path == "stream"
+    tensor_ok = wl.d % 128 == 0 and wl.f % 128 == 0     # the library's own choice, restated for the work model
+    stream_path = (wl.T <= (32 if tensor_ok else 64) and wl.d % 64 == 0 and wl.f % 64 == 0) \
+        if args.path == "auto" else args.path == "stream"
 
     def step_device():
         if is_stack:

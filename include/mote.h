@@ -54,7 +54,8 @@ enum { MOTE_SHARED_BF16 = 16, MOTE_SHARED_INT8 = 8, MOTE_SHARED_INT4 = 4 };
  *   TENSOR  d % 128 == 0 and f % 128 == 0: tcgen05 GEMMs (int8 x 2-bit routed, bf16 shared; an
  *           RTN-coded shared expert is expanded to bf16 on the way, see mote_layer_workspace_bytes)
  *   SIMT    any d, f that are multiples of 16: CUDA-core GEMMs
- * AUTO takes the first of these whose conditions hold. */
+ * AUTO takes STREAM up to 32 tokens (up to 64 where TENSOR's conditions do not hold), then TENSOR,
+ * then SIMT. */
 enum { MOTE_PATH_AUTO = 0, MOTE_PATH_SIMT = 1, MOTE_PATH_TENSOR = 2, MOTE_PATH_STREAM = 3 };
 
 const char* mote_status_string(mote_status_t st);

@@ -40,6 +40,7 @@ struct Plan {
 // layer to bf16 in the workspace (one streaming pass) and runs the plain bf16 GEMMs on them; below,
 // the GEMM expands the codes tile by tile in shared memory (less weight traffic, more work per row tile).
 constexpr int64_t kExpandMinTokens = 768;
+constexpr int64_t kStreamAutoMaxTokens = 32;
 
 static Plan make_plan(int d, int f, int E, int k, int64_t T) {
   Plan p{};
@@ -262,7 +263,11 @@ extern "C" mote_status_t mote_moe_forward(const mote_layer_t* L, const void* x, 
   const bool tensor_ok = (d % 128 == 0) && (f % 128 == 0);
   const bool stream_ok = decode_stream_supported(d, f, E, k, T);
   int path = L->path;
-  if (path == MOTE_PATH_AUTO) path = stream_ok ? MOTE_PATH_STREAM : tensor_ok ? MOTE_PATH_TENSOR : MOTE_PATH_SIMT;
+  // AUTO: the weight stream up to 32 tokens (beyond that its eight-column-tile kernels run at low
+  // occupancy and the tcgen05 GEMMs, with the shared down projection split along K, are faster)
+  if (path == MOTE_PATH_AUTO)
+    path = (stream_ok && (T <= kStreamAutoMaxTokens || !tensor_ok)) ? MOTE_PATH_STREAM
+           : tensor_ok ? MOTE_PATH_TENSOR : MOTE_PATH_SIMT;
   if (path == MOTE_PATH_STREAM && !stream_ok) return MOTE_ERR_SHAPE;
   if (path == MOTE_PATH_TENSOR && !tensor_ok) return MOTE_ERR_SHAPE;
   const bool tensor = (path == MOTE_PATH_TENSOR);

@@ -34,7 +34,7 @@ def test_rms_norm(mote, T, d):
 
 
 @pytest.mark.parametrize("rms_eps,shared_bits", [(1e-6, 16), (0.0, 16), (1e-6, 8), (1e-6, 4)])
-@pytest.mark.parametrize("T", [1, 40, 150])          # decode path (1, 40) and tensor-core path (150)
+@pytest.mark.parametrize("T", [1, 24, 40, 150])      # decode path (1, 24) and tensor-core path (40: K-split shared down; 150)
 def test_small_stack_per_layer_parity(mote, T, rms_eps, shared_bits):
     n_layers = 5
     wl = synth.custom("stack", 128, 256, 4, 2, T, 4100, n_layers=n_layers, w_std=0.08)
@@ -101,3 +101,36 @@ def test_stack_argument_errors(mote):
     assert lib.mote_stack_forward(arr, 1, eps, fake, 4, fake, None, fake, 1 << 20, None) == 2    # out aliases x
     assert lib.mote_stack_forward(arr, 1, C.c_float(-1.0), fake, 4, C.c_void_p(0x2000), None, fake, 1 << 20, None) == 2
     assert lib.mote_rms_norm(fake, 4, 12, eps, fake, None) == 2 and lib.mote_rms_norm(None, 4, 16, eps, fake, None) == 1
+
+
+@pytest.mark.parametrize("T", [1, 200])
+def test_stack_forward_can_be_captured_in_a_cuda_graph(mote, T):
+    # the library only enqueues on the caller's stream: a captured step replays to the same bits
+    n_layers = 3
+    wl = synth.custom("graph", 128, 256, 4, 2, T, 4200, n_layers=n_layers, w_std=0.08)
+    layers = [mote.MoteLayer.from_master(synth.master_layer(wl, layer=l)) for l in range(n_layers)]
+    stack = mote.MoteStack(layers)
+    x = bf16_tensor(synth.tokens(wl))
+    out = torch.empty_like(x)
+    want = mote.mote_stack_forward(stack, x).clone()          # also the warm-up (first-call set-up, workspace)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        mote.mote_stack_forward(stack, x, out=out)
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        mote.mote_stack_forward(stack, x, out=out)
+    for _ in range(3):
+        out.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(out, want)
+    # new input in the same buffer, same graph
+    x2 = bf16_tensor(synth.tokens(wl, stream=1))
+    want2 = mote.mote_stack_forward(stack, x2).clone()
+    x.copy_(x2)
+    graph.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(out, want2)
