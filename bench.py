@@ -104,7 +104,8 @@ NCU_TRAFFIC_BYTES = {("c2", "gateup_ternary"): 42.73e6, ("c4", "gateup_ternary")
                      ("c3-1", "gateup_ternary"): 69.85e6}
 
 
-def stage_work(wl: synth.Workload, stage: str, stream_path: bool, experts_touched: float, shared_bits: int = 16):
+def stage_work(wl: synth.Workload, stage: str, stream_path: bool, experts_touched: float, shared_bits: int = 16,
+               peaks: dict | None = None):
     """Algorithmic work of one launch of a stage: (amount, kind), kind 'int8' | 'bf16' | 'bytes'.
     On the decode path the gate/up and down stages each cover the routed AND the shared expert and
     are bound by the weight bytes they stream: 2-bit codes of the experts that received tokens plus
@@ -116,14 +117,19 @@ def stage_work(wl: synth.Workload, stage: str, stream_path: bool, experts_touche
             return experts_touched * 2 * f * d / 4 + 2.0 * f * d * sh_bytes, "bytes"
         if stage == "down_ternary":
             return experts_touched * f * d / 4 + f * d * sh_bytes, "bytes"
-    if stage == "gateup_ternary":
-        return 2.0 * P * d * 2 * f, "int8"
-    if stage == "down_ternary":
-        return 2.0 * P * f * d, "int8"
-    if stage == "shared_gateup":
-        return 2.0 * T * d * 2 * f, "bf16"
-    if stage == "shared_down":
-        return 2.0 * T * f * d, "bf16"
+    # the four GEMMs: tensor work, or -- with few tokens -- the bytes they must move, whichever takes
+    # longer at the peaks (a short prefill streams the weights once and is bound by that)
+    gemm = {"gateup_ternary": (2.0 * P * d * 2 * f, "int8", experts_touched * 2 * f * d / 4 + P * d + P * f * 2.0),
+            "down_ternary": (2.0 * P * f * d, "int8", experts_touched * f * d / 4 + P * f + P * d * 4.0),
+            "shared_gateup": (2.0 * T * d * 2 * f, "bf16", 2.0 * f * d * sh_bytes + T * d * 2.0 + T * f * 2.0),
+            "shared_down": (2.0 * T * f * d, "bf16", f * d * sh_bytes + T * f * 2.0 + T * d * 2.0)}
+    if stage in gemm:
+        ops, kind, nbytes = gemm[stage]
+        if peaks is not None:
+            t_ops = ops / (peaks["bf16_tflops"] * 1e12 * (NOMINAL_INT8_OVER_BF16 if kind == "int8" else 1.0))
+            if nbytes / (peaks["hbm_gbs"] * 1e9) > t_ops:
+                return nbytes, "bytes"
+        return ops, kind
     if stage == "quant_x":
         return T * d * 2.0 + P * d * 1.0, "bytes"
     if stage == "quant_h":
@@ -317,7 +323,7 @@ def run_ours(args):
     tokens_per_s = job_tokens_per_s(world, wl.T, args.steps, total_ms)
     decode = wl.T <= 64
     dom = max(stage_ms, key=stage_ms.get)
-    work, kind = stage_work(wl, dom, stream_path, experts_touched, args.shared_bits)
+    work, kind = stage_work(wl, dom, stream_path, experts_touched, args.shared_bits, peaks)
     dur_s = stage_ms[dom] * 1e-3 / len(layers)          # average duration of one launch of that kernel
     if kind == "bytes":
         roof = dict(bound="hbm", achieved=work / dur_s / 1e9, peak=peaks["hbm_gbs"], unit="GB/s")
