@@ -91,6 +91,20 @@ __global__ void __launch_bounds__(256) decode_prologue_kernel(DecodePrologueArgs
   const uint4* src = reinterpret_cast<const uint4*>(a.x + int64_t(t) * d);
   pdl_trigger();                         // the gate/up kernel may start on the shared expert right away
 
+  // The router weights do not depend on the token: the first pass's rows for this thread's first
+  // unit are requested now, and the later passes' rows are pulled into L2, so that their latency
+  // runs under the absmax / Q_a(x) phase instead of after it.
+  float4 wp0[8], wq0[8];
+  if (tid < n_vec) {
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+      const float4* wr = reinterpret_cast<const float4*>(a.Wr + int64_t(min(c, a.E - 1)) * d) + 2 * tid;
+      wp0[c] = wr[0]; wq0[c] = wr[1];
+    }
+    for (int e = 8; e < a.E; ++e)
+      asm volatile("prefetch.global.L2 [%0];" ::"l"(a.Wr + int64_t(e) * d + 8 * tid));
+  }
+
   float amax = 0.0f;
   for (int v = tid; v < n_vec; v += 256) {
     const uint4 r = src[v];
@@ -142,10 +156,15 @@ __global__ void __launch_bounds__(256) decode_prologue_kernel(DecodePrologueArgs
       const float xv[8] = {bf16_lo(r.x), bf16_hi(r.x), bf16_lo(r.y), bf16_hi(r.y),
                            bf16_lo(r.z), bf16_hi(r.z), bf16_lo(r.w), bf16_hi(r.w)};
       float4 wp[8], wq[8];
+      if (e0 == 0 && v == tid) {
 #pragma unroll
-      for (int c = 0; c < 8; ++c) {
-        const float4* wr = reinterpret_cast<const float4*>(a.Wr + int64_t(min(e0 + c, a.E - 1)) * d) + 2 * v;
-        wp[c] = wr[0]; wq[c] = wr[1];
+        for (int c = 0; c < 8; ++c) { wp[c] = wp0[c]; wq[c] = wq0[c]; }
+      } else {
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          const float4* wr = reinterpret_cast<const float4*>(a.Wr + int64_t(min(e0 + c, a.E - 1)) * d) + 2 * v;
+          wp[c] = wr[0]; wq[c] = wr[1];
+        }
       }
 #pragma unroll
       for (int c = 0; c < 8; ++c) {
