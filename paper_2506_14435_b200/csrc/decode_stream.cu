@@ -242,7 +242,31 @@ __global__ void __launch_bounds__(256) decode_prologue_kernel(DecodePrologueArgs
           a.topk_w[t * k + j] = ex[j] / denom;
         }
     }
+    if (a.T == 1) {
+      // one token: its k pairs are grouped right here (every lane holds the selection), without
+      // the round trips of the arrival counter
+      int mine = 0;
+#pragma unroll
+      for (int j = 0; j < MOTE_MAX_TOPK; ++j)
+        if (j < k && lane == j) mine = sel_i[j];
+      int rank = 0;
+      for (int e = lane; e <= E; e += 32) {
+        int c = 0;
+#pragma unroll
+        for (int j = 0; j < MOTE_MAX_TOPK; ++j)
+          if (j < k) c += sel_i[j] < e ? 1 : 0;
+        a.offsets[e] = c;
+      }
+#pragma unroll
+      for (int j = 0; j < MOTE_MAX_TOPK; ++j)
+        if (j < k) rank += sel_i[j] < mine ? 1 : 0;
+      if (lane < k) {
+        a.perm[lane] = rank;
+        a.inv[rank] = lane;
+      }
+    }
   }
+  if (a.T == 1) return;
 
   // the CTA that finishes last sees every token's selection and groups the pairs by expert
   __threadfence();
