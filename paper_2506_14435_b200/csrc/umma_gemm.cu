@@ -123,8 +123,9 @@ __device__ __forceinline__ void decode_item(const UmmaArgs& a, int item, int n_m
   tile = a.tiles[1 + m_tile];
 }
 // pipeline steps [kb, ke) of an item, and which split it is
+template <bool kGateUp>
 __device__ __forceinline__ int item_k_range(const UmmaArgs& a, int item, int& kb, int& ke) {
-  if (a.k_splits <= 1) { kb = 0; ke = a.k_steps; return 0; }
+  if (kGateUp || a.k_splits <= 1) { kb = 0; ke = a.k_steps; return 0; }
   const int split = (item / a.n_ntiles) % a.k_splits;
   kb = split * a.k_steps / a.k_splits;
   ke = (split + 1) * a.k_steps / a.k_splits;
@@ -180,7 +181,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
   const uint32_t tmem_base = bars->tmem_base;
   pdl_wait();                              // set-up above overlaps the tail of the kernel before this one
   const int n_mtiles = a.tiles[0].x;
-  const int n_items = n_mtiles * a.n_ntiles * a.k_splits;
+  const int n_items = n_mtiles * a.n_ntiles * (TR::kGateUp ? 1 : a.k_splits);
 
   if (warp == 0) {
     // ---------------------------------------------------------------- token-operand producer
@@ -192,7 +193,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
         decode_item<TR::kGateUp>(a, item, n_mtiles, tile, n_tile);
         const int b_row = (a.b_rows_per_expert ? tile.x * a.b_rows_per_expert : 0) + n_tile * (TR::kGateUp ? a.bn / 2 : a.bn);
         int kb, ke;
-        item_k_range(a, item, kb, ke);
+        item_k_range<TR::kGateUp>(a, item, kb, ke);
         for (int ks = kb; ks < ke; ++ks) {
           if (!(ok = mbar_wait(smem_u32(&bars->empty[stage]), phase ^ 1, abort_flag))) break;
           const uint32_t bar = smem_u32(&bars->full_a[stage]);
@@ -228,7 +229,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
         decode_item<TR::kGateUp>(a, item, n_mtiles, tile, n_tile);
         const int b_row = tile.x * a.b_rows_per_expert + n_tile * (TR::kGateUp ? a.bn / 2 : a.bn);
         int kb, ke;
-        item_k_range(a, item, kb, ke);
+        item_k_range<TR::kGateUp>(a, item, kb, ke);
         for (int ks = kb; ks < ke; ++ks) {
           if (!(ok = mbar_wait(smem_u32(&bars->empty_p[stage]), phase ^ 1, abort_flag))) break;
           const uint32_t bar = smem_u32(&bars->full_p[stage]);
@@ -260,7 +261,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * 256;
         int kb, ke;
-        item_k_range(a, item, kb, ke);
+        item_k_range<TR::kGateUp>(a, item, kb, ke);
         for (int ks = kb; ks < ke; ++ks) {
           if (!(ok = mbar_wait(smem_u32(&bars->full_a[stage]), phase, abort_flag))) break;
           if (TR::kUnpack)
@@ -292,7 +293,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
       const int n_chunks = a.bn * (TR::kCodeRowBytes / 16);   // chunks of 16 code bytes, spread over 128 threads
       for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x) {
         int kb, ke;
-        item_k_range(a, item, kb, ke);
+        item_k_range<TR::kGateUp>(a, item, kb, ke);
         for (int ks = kb; ks < ke; ++ks, ++step) {
           if ((step & 1u) == (uint32_t)group) {
             ok = mbar_wait(smem_u32(&bars->full_p[pstage]), pphase, abort_flag) &&
@@ -368,7 +369,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
       int4 tile; int n_tile;
       decode_item<TR::kGateUp>(a, item, n_mtiles, tile, n_tile);
       int kb_, ke_;
-      const int split = item_k_range(a, item, kb_, ke_);
+      const int split = item_k_range<TR::kGateUp>(a, item, kb_, ke_);
       const int buf = local & 1;
       const uint32_t use = (uint32_t)(local >> 1);
       ok = mbar_wait(smem_u32(&bars->tmem_full[buf]), use & 1, abort_flag);
