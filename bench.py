@@ -100,8 +100,8 @@ class ClockSampler:
 
 # ncu dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the captures
 # summarised under profiles/ (null once the kernel has changed since, or where no capture exists)
-NCU_TRAFFIC_BYTES = {("c2", "gateup_ternary"): 42.73e6, ("c4", "gateup_ternary"): 587.09e6,
-                     ("c3-1", "gateup_ternary"): 69.85e6}
+NCU_TRAFFIC_BYTES = {("c2", "gateup_ternary"): 42.88e6, ("c4", "gateup_ternary"): 610.09e6,
+                     ("c3-1", "gateup_ternary"): 69.92e6}
 
 
 def stage_work(wl: synth.Workload, stage: str, stream_path: bool, experts_touched: float, shared_bits: int = 16,
