@@ -650,7 +650,14 @@ mote_status_t launch_ternary_umma(const TernaryGemmArgs& g, bool gateup, const i
                                   cudaStream_t stream, bool pdl) {
   if (g.P == 0) return MOTE_OK;
   CUtensorMap ta, tb0, tb1;
-  const int bn = gateup ? 256 : pick_bn(g.N);
+  int bn = gateup ? 256 : pick_bn(g.N);
+  // a down projection with few row tiles: 128-wide tiles double the items (the weights are the
+  // traffic here, and they are read once either way)
+  if (!gateup && bn > 128) {
+    int dev = 0, sms = 148;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (max_mtiles * (g.N / bn) * 2 <= sms) bn = 128;
+  }
   if (!make_map_2d(&ta, g.qa, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)g.P, (uint64_t)g.K, 128, 128,
                    CU_TENSOR_MAP_SWIZZLE_128B))
     return MOTE_ERR_CUDA;
