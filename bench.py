@@ -387,11 +387,16 @@ def cpu_baseline(wl, master, x_bits, budget_s: float, n_tokens: int | None = Non
     rate = n0 / max(time.perf_counter() - t0, 1e-6)
     n = n_tokens or int(min(wl.T, max(n0, rate * budget_s)))
     sub = np.arange(n)
-    t0 = time.perf_counter()
-    O.moe_forward(layer_or, x_bits, token_subset=sub)
-    dt = time.perf_counter() - t0
-    return {"value": n / dt, "unit": "tokens/s", "cores": torch.get_num_threads(), "kind": "oracle",
-            "sample": f"first {n} of {wl.T} tokens of {wl.name} (routing for all tokens), {dt:.2f} s",
+    passes, dt = 0, 0.0
+    while True:                                          # whole passes over the sample until the budget is used
+        t0 = time.perf_counter()
+        O.moe_forward(layer_or, x_bits, token_subset=sub)
+        dt += time.perf_counter() - t0
+        passes += 1
+        if dt >= 0.8 * budget_s or dt + dt / passes > 2.5 * budget_s:
+            break
+    return {"value": n * passes / dt, "unit": "tokens/s", "cores": torch.get_num_threads(), "kind": "oracle",
+            "sample": f"first {n} of {wl.T} tokens of {wl.name} (routing for all tokens), {passes} pass(es), {dt:.2f} s",
             "seconds": dt}
 
 
