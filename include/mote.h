@@ -64,8 +64,9 @@ const char* mote_status_string(mote_status_t st);
  * mote_ternarize_pack -- absmean ternary weight quantizer and INT2 packing (Eq. 7, 9, 10; storage
  * per Section 3.1).  Offline step, once per matrix.
  *
- *   alpha  = max( fl32( (exact sum of |w|) / (m*n) ), 1e-5 )   the sum is exact (integer
- *            accumulation of fp32 significands), so alpha does not depend on thread order
+ *   alpha  = max( fl32( fl64(exact sum of |w|) / (m*n) ), 1e-5 )   the sum is exact (integer
+ *            accumulation of fp32 significands), so alpha does not depend on thread order; it is
+ *            rounded once to fp64, divided in fp64 and the quotient rounded to fp32
  *   code   = clamp( rint( w / alpha ), -1, 1 )                 true fp32 division, ties to even
  *   packed : m * n/4 bytes; stored value u = code + 1; 4 consecutive elements of a row per byte,
  *            element j in bits [2*(j%4), 2*(j%4)+1]
@@ -91,15 +92,19 @@ mote_status_t mote_ternarize_pack(const void* W, int w_dtype, int64_t m, int64_t
  * device-wide synchronisation an allocation may imply.
  * The 256 exponent bins (2 KiB) that the exact sum of |w| needs live in a device array inside the
  * library image, so every GPU that loads the library carries those 2 KiB until the process ends.
- * The call itself makes no device allocation of any kind; it issues one memset, three kernels.
+ * The call itself asks for no device memory; it issues one memset and three kernels.  (The very
+ * first use of the library on a device may make the CUDA runtime load the library's code there;
+ * that happens once, is not specific to this call, and a caller that must avoid it warms up once
+ * at start-up.)
  *
  *   W, w_dtype, m, n, packed, alpha, stream    exactly as mote_ternarize_pack
  *
  * Limits and rules
  *   - m*n <= MOTE_STATIC_MAX_ELEMENTS (2^31, e.g. a 32768 x 65536 matrix); beyond that the call
  *     returns MOTE_ERR_TOO_LARGE and launches nothing.  Use mote_ternarize_pack for larger ones.
- *   - The first call on each device looks up the device address of the array (a host-side query,
- *     no allocation).  Make that first call outside any stream capture.
+ *   - The first call on each device looks up the device address of the array (a host-side query)
+ *     and keeps it for the life of the process; make that first call outside any stream capture.
+ *     The kept address does not survive cudaDeviceReset.
  *   - All calls on one device share the one array, and it keeps what the last call left in it;
  *     each call clears it on `stream` before use.  Two calls that can overlap on the GPU (issued
  *     on different streams without an ordering between them, or from two host threads) race on
@@ -309,10 +314,23 @@ mote_status_t mote_moe_forward_profile(const mote_layer_t* L, const void* x_bf16
                                        const void* residual_bf16, int64_t T, void* out_bf16,
                                        void* ws, size_t ws_bytes, void* stream, float* stage_ms_host);
 
-/* Reads (and clears) the device status word kept at the start of a workspace after the stream has
- * been synchronised by the caller: MOTE_OK, or MOTE_ERR_DEVICE_TIMEOUT if a kernel gave up a
- * bounded wait.  Synchronises the stream itself. */
+/* Reads (and clears) the device status word kept in the first 4 bytes of a workspace: MOTE_OK, or
+ * MOTE_ERR_DEVICE_TIMEOUT if a kernel gave up a bounded wait (every device-side wait of the GEMM
+ * kernels has a time limit; a CTA whose wait runs out stops working, lets copies in flight land,
+ * releases its tensor memory, raises this word and returns normally, so the context stays usable
+ * and the output of that call is invalid).  Synchronises the stream itself.
+ * The word is cleared at the start of every mote_moe_forward / mote_moe_forward_host call and once
+ * at the start of mote_stack_forward (not between its layers), so it reports the last such call. */
 mote_status_t mote_device_status(void* ws, void* stream);
+
+/* Diagnostic for the mechanism above (no counterpart in the paper): enqueues one thread block that
+ * waits, with the GEMM kernels' own bounded wait, on a barrier nothing ever arrives at.  After about
+ * limit_ns nanoseconds the wait gives up and the block raises the status word in ws[0..3] exactly
+ * as a GEMM would; nothing faults and nothing hangs.  mote_device_status(ws) then returns
+ * MOTE_ERR_DEVICE_TIMEOUT once, and MOTE_OK afterwards.
+ *   ws        device memory, at least 4 bytes, 256-B aligned (any workspace will do)
+ *   limit_ns  1 000 .. 100 000 000 (1 us .. 100 ms); outside -> ERR_SHAPE */
+mote_status_t mote_selftest_bounded_wait(void* ws, uint64_t limit_ns, void* stream);
 
 /* Number of kernels the last mote_moe_forward call on this thread enqueued. */
 int mote_last_launch_count(void);

@@ -81,6 +81,8 @@ lib.mote_moe_forward_profile.argtypes = [C.POINTER(mote_layer_t), C.c_void_p, C.
                                          C.c_void_p, C.c_size_t, C.c_void_p, C.POINTER(C.c_float)]
 lib.mote_device_status.restype = C.c_int
 lib.mote_device_status.argtypes = [C.c_void_p, C.c_void_p]
+lib.mote_selftest_bounded_wait.restype = C.c_int
+lib.mote_selftest_bounded_wait.argtypes = [C.c_void_p, C.c_uint64, C.c_void_p]
 lib.mote_last_launch_count.restype = C.c_int
 lib.mote_last_launch_count.argtypes = []
 

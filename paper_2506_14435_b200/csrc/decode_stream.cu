@@ -934,13 +934,7 @@ bool decode_stream_supported(int d, int f, int E, int k, int64_t T) {
 // phase 0: prologue, 1: gate/up, 2: down
 mote_status_t launch_decode_stream(const DecodeStreamArgs& p, int phase, cudaStream_t stream) {
   const int T = (int)p.T, d = p.d, f = p.f, E = p.E, k = p.k;
-  static int sms = 0;
-  if (sms == 0) {
-    int dev = 0, n = 148;
-    MOTE_CUDA_OK(cudaGetDevice(&dev));
-    MOTE_CUDA_OK(cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev));
-    sms = n;
-  }
+  const int sms = device_sm_count();
   const int ntb = T <= 8 ? 1 : T <= 16 ? 2 : T <= 32 ? 4 : 8;
 
   if (phase == 0) {
@@ -949,11 +943,8 @@ mote_status_t launch_decode_stream(const DecodeStreamArgs& p, int phase, cudaStr
     pa.Wr = p.Wr; pa.bias = p.router_bias; pa.topk_idx = p.topk_idx; pa.topk_w = p.topk_w; pa.qx = p.qx;
     pa.beta_x = p.beta_x; pa.rowsum_x = p.rowsum_x; pa.beta_h_bits = reinterpret_cast<uint32_t*>(p.beta_h);
     pa.rowsum_h = p.rowsum_h; pa.counter = p.counter; pa.offsets = p.offsets; pa.perm = p.perm; pa.inv = p.inv;
-    static bool attr_set = false;
-    if (!attr_set) {
-      MOTE_CUDA_OK(cudaFuncSetAttribute(decode_prologue_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 32768));
-      attr_set = true;
-    }
+    static PerDeviceOnce prologue_attr;
+    MOTE_CUDA_OK(set_max_dynamic_smem(prologue_attr, decode_prologue_kernel, 32768));
     decode_prologue_kernel<<<T, 256, size_t(d) * 2, stream>>>(pa);
     ++g_launch_count;
     MOTE_LAUNCH_OK();
@@ -1003,13 +994,10 @@ mote_status_t launch_decode_stream(const DecodeStreamArgs& p, int phase, cudaStr
   const int max_items = tiles + std::min<int>(E, T * k) * tiles;
   const int grid = std::min(max_items, sms * 3);
   const size_t smem = size_t(kDownWarps) * ntb * 4 * 32 * sizeof(float);
-  static bool down_attr_set = false;
-  if (!down_attr_set) {
-    MOTE_CUDA_OK(cudaFuncSetAttribute(decode_down_kernel<8, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 65536));
-    MOTE_CUDA_OK(cudaFuncSetAttribute(decode_down_kernel<8, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 65536));
-    MOTE_CUDA_OK(cudaFuncSetAttribute(decode_down_kernel<8, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 65536));
-    down_attr_set = true;
-  }
+  static PerDeviceOnce down_attr16, down_attr8, down_attr4;
+  MOTE_CUDA_OK(set_max_dynamic_smem(down_attr16, decode_down_kernel<8, 16>, 65536));
+  MOTE_CUDA_OK(set_max_dynamic_smem(down_attr8, decode_down_kernel<8, 8>, 65536));
+  MOTE_CUDA_OK(set_max_dynamic_smem(down_attr4, decode_down_kernel<8, 4>, 65536));
 #define MOTE_DN_LAUNCH(NTB_, BITS_) \
   MOTE_CUDA_OK(launch_pdl(decode_down_kernel<NTB_, BITS_>, dim3(grid), dim3(kDownWarps * 32), smem, stream, da))
 #define MOTE_DN_BITS(NTB_)                                 \

@@ -12,6 +12,11 @@ namespace mote {
 
 thread_local int g_launch_count = 0;
 
+// Set while mote_stack_forward runs its layers: the stack clears the device status word once, at
+// its start, and the layer calls inside it leave the word alone, so that a bounded wait that ran
+// out in ANY layer is still there when the caller reads mote_device_status after the stack.
+static thread_local bool g_keep_status = false;
+
 // Optional per-stage CUDA events (mote_moe_forward_profile): event i is recorded on the launch
 // stream after stage i has been enqueued, event 0 before the first stage.
 struct StageTimer {
@@ -23,9 +28,9 @@ static inline void stage_mark(int i, cudaStream_t stream) {
   if (g_timer.active) cudaEventRecord(g_timer.ev[i], stream);
 }
 
-// Head of the workspace, cleared at the start of every call: [0] device status word, [1] arrival
-// counter of the decode prologue, from byte 256 on the per-tile arrival counters of the decode
-// path's down kernel (d / 16 <= 2048 words).
+// Head of the workspace: [0] device status word (cleared at the start of every top-level call),
+// [1] arrival counter of the decode prologue, from byte 256 on the per-tile arrival counters of the
+// decode path's down kernel (d / 16 <= 2048 words); the counters are cleared by every layer call.
 constexpr size_t kStatusBytes = 256 + 2048 * 4;
 
 struct Plan {
@@ -206,6 +211,13 @@ extern "C" mote_status_t mote_device_status(void* ws, void* stream_) {
   return MOTE_OK;
 }
 
+extern "C" mote_status_t mote_selftest_bounded_wait(void* ws, uint64_t limit_ns, void* stream_) {
+  if (!ws) return MOTE_ERR_NULL;
+  if ((reinterpret_cast<uintptr_t>(ws) & 255u) != 0) return MOTE_ERR_ALIGN;
+  if (limit_ns < 1000ull || limit_ns > 100000000ull) return MOTE_ERR_SHAPE;
+  return launch_bounded_wait_selftest(static_cast<uint32_t*>(ws), limit_ns, static_cast<cudaStream_t>(stream_));
+}
+
 extern "C" mote_status_t mote_moe_forward(const mote_layer_t* L, const void* x, const void* residual, int64_t T,
                                           void* out, const mote_taps_t* taps, void* ws, size_t ws_bytes,
                                           void* stream_) {
@@ -275,7 +287,8 @@ extern "C" mote_status_t mote_moe_forward(const mote_layer_t* L, const void* x, 
 
   if (path == MOTE_PATH_STREAM) {
     // status word, the prologue's arrival counter, the down kernel's tile counters
-    MOTE_CUDA_OK(cudaMemsetAsync(status, 0, 256 + size_t(d / 16) * 4, stream));
+    const size_t keep = g_keep_status ? 4 : 0;
+    MOTE_CUDA_OK(cudaMemsetAsync(reinterpret_cast<char*>(status) + keep, 0, 256 + size_t(d / 16) * 4 - keep, stream));
     stage_mark(0, stream);
     DecodeStreamArgs ds{};
     ds.x = x; ds.T = T; ds.d = d; ds.f = f; ds.E = E; ds.k = k; ds.norm_topk = L->norm_topk;
@@ -325,7 +338,7 @@ extern "C" mote_status_t mote_moe_forward(const mote_layer_t* L, const void* x, 
   }
 
   mote_status_t st;
-  MOTE_CUDA_OK(cudaMemsetAsync(status, 0, 4, stream));
+  if (!g_keep_status) MOTE_CUDA_OK(cudaMemsetAsync(status, 0, 4, stream));
   stage_mark(0, stream);
   // S1 router, S2 dispatch
   // block-wise dispatch: the tensor-core router (d % 32 == 0) leaves per-block expert counts, a small
@@ -495,6 +508,8 @@ extern "C" mote_status_t mote_stack_forward(const mote_layer_t* layers, int n_la
   void* normed = ping + 2 * slab;
   int launches = 0;
   const void* res = x;                                 // residual stream x_{l-1}
+  MOTE_CUDA_OK(cudaMemsetAsync(ws, 0, 4, stream));     // device status word: once for the whole stack
+  struct KeepStatus { KeepStatus() { g_keep_status = true; } ~KeepStatus() { g_keep_status = false; } } keep_status;
   for (int l = 0; l < n_layers; ++l) {
     void* dst = (l == n_layers - 1) ? out : static_cast<void*>(ping + size_t(l & 1) * slab);
     if (layer_inputs)

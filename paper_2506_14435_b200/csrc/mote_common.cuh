@@ -4,6 +4,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "mote.h"
 
 #define MOTE_CUDA_OK(expr)                                   \
@@ -74,6 +76,50 @@ constexpr float kEpsScale = 1e-5f;  // lower clamp of alpha (Eq. 9) and beta (Eq
 
 static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 static inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// ---------------------------------------------------------------------------------------------
+// Per-device host state.  Function attributes (the dynamic shared memory limit) and the SM count
+// belong to a device, not to the process: a process that drives several GPUs must set / query them
+// once on each.  Device ordinals beyond kMaxDevices are served without caching.
+// ---------------------------------------------------------------------------------------------
+constexpr int kMaxDevices = 64;
+
+static inline int current_device() {
+  int dev = 0;
+  return cudaGetDevice(&dev) == cudaSuccess ? dev : -1;
+}
+
+// SM count of the current device (148 if the query fails)
+static inline int device_sm_count() {
+  static std::atomic<int> cache[kMaxDevices];
+  const int dev = current_device();
+  if (dev >= 0 && dev < kMaxDevices) {
+    const int c = cache[dev].load(std::memory_order_relaxed);
+    if (c > 0) return c;
+  }
+  int n = 148;
+  if (dev < 0 || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return 148;
+  if (dev < kMaxDevices) cache[dev].store(n, std::memory_order_relaxed);
+  return n;
+}
+
+// One flag per device for a set-up step that must run once on each (setting it twice is harmless,
+// so a relaxed flag is enough).  Declare one `static PerDeviceOnce` beside the step it guards.
+struct PerDeviceOnce {
+  std::atomic<bool> done[kMaxDevices];
+  bool needed(int dev) const { return dev < 0 || dev >= kMaxDevices || !done[dev].load(std::memory_order_acquire); }
+  void mark(int dev) { if (dev >= 0 && dev < kMaxDevices) done[dev].store(true, std::memory_order_release); }
+};
+
+// Raises the dynamic shared memory limit of `kernel` on the current device, once per device.
+template <typename K>
+static inline cudaError_t set_max_dynamic_smem(PerDeviceOnce& once, K kernel, int bytes) {
+  const int dev = current_device();
+  if (!once.needed(dev)) return cudaSuccess;
+  const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess) once.mark(dev);
+  return e;
+}
 
 // Counts kernel launches of the current forward call (host side, per thread).
 extern thread_local int g_launch_count;

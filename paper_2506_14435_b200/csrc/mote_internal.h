@@ -97,6 +97,9 @@ mote_status_t launch_shared_umma(const void* act, const SharedMat& w0, const Sha
                                  int64_t T, int K, int N, void* out, const int4* tiles, int max_mtiles,
                                  uint32_t* status, const CombineArgs* comb, cudaStream_t stream, bool pdl = false,
                                  int k_splits = 1);
+// Diagnostic: one CTA waits on an mbarrier that nothing arrives at, with the GEMM kernels' bounded
+// wait and teardown; after limit_ns it raises *status and returns.
+mote_status_t launch_bounded_wait_selftest(uint32_t* status, uint64_t limit_ns, cudaStream_t stream);
 constexpr int64_t kMaxPartialRows = 4096;
 int shared_down_k_splits(int64_t T, int N, int K);
 

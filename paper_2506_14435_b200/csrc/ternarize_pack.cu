@@ -148,26 +148,18 @@ __global__ void __launch_bounds__(256) pack_codes_kernel(const void* __restrict_
 
 }  // namespace mote
 
-extern "C" size_t mote_ternarize_workspace_bytes(void) { return mote::kBins * sizeof(unsigned long long); }
+namespace mote {
 
-extern "C" mote_status_t mote_ternarize_pack(const void* W, int w_dtype, int64_t m, int64_t n,
-                                             uint8_t* packed, float* alpha, void* ws, size_t ws_bytes,
-                                             void* stream_) {
-  using namespace mote;
-  if (!W || !packed || !alpha || !ws) return MOTE_ERR_NULL;
-  if (w_dtype != MOTE_DTYPE_F32 && w_dtype != MOTE_DTYPE_BF16) return MOTE_ERR_DTYPE;
-  if (m <= 0 || n <= 0 || (n % 16) != 0) return MOTE_ERR_SHAPE;
-  if (m >= (int64_t(1) << 38) / n) return MOTE_ERR_SHAPE;
-  if (!aligned16(W) || !aligned16(packed) || !aligned16(ws)) return MOTE_ERR_ALIGN;
-  if (ws_bytes < mote_ternarize_workspace_bytes()) return MOTE_ERR_WORKSPACE;
-  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-  auto* bins = static_cast<unsigned long long*>(ws);
-  const int64_t total = m * n;
+// The quantizer's launch sequence on exponent bins that the caller owns (a workspace, or the
+// library's built-in array): clear the bins, exact sum of |w|, alpha, codes.
+static mote_status_t ternarize_with_bins(const void* W, int w_dtype, int64_t total, uint8_t* packed, float* alpha,
+                                         unsigned long long* bins, cudaStream_t stream) {
   const int64_t n_vec = total / 4, n_words = total / 16;
-  MOTE_CUDA_OK(cudaMemsetAsync(bins, 0, mote_ternarize_workspace_bytes(), stream));
+  // whatever the bins held before (an earlier call's sums, or nothing defined) must go
+  MOTE_CUDA_OK(cudaMemsetAsync(bins, 0, kBins * sizeof(unsigned long long), stream));
   const int threads = 256;
-  int blocks_a = (int)std::min<int64_t>((n_vec + threads - 1) / threads, 148 * 8);
-  int blocks_c = (int)std::min<int64_t>((n_words + threads - 1) / threads, 148 * 16);
+  const int blocks_a = (int)std::min<int64_t>((n_vec + threads - 1) / threads, 148 * 8);
+  const int blocks_c = (int)std::min<int64_t>((n_words + threads - 1) / threads, 148 * 16);
   if (w_dtype == MOTE_DTYPE_BF16)
     abs_sum_bins_kernel<true><<<blocks_a, threads, 0, stream>>>(W, n_vec, bins);
   else
@@ -183,6 +175,24 @@ extern "C" mote_status_t mote_ternarize_pack(const void* W, int w_dtype, int64_t
   return MOTE_OK;
 }
 
+}  // namespace mote
+
+extern "C" size_t mote_ternarize_workspace_bytes(void) { return mote::kBins * sizeof(unsigned long long); }
+
+extern "C" mote_status_t mote_ternarize_pack(const void* W, int w_dtype, int64_t m, int64_t n,
+                                             uint8_t* packed, float* alpha, void* ws, size_t ws_bytes,
+                                             void* stream_) {
+  using namespace mote;
+  if (!W || !packed || !alpha || !ws) return MOTE_ERR_NULL;
+  if (w_dtype != MOTE_DTYPE_F32 && w_dtype != MOTE_DTYPE_BF16) return MOTE_ERR_DTYPE;
+  if (m <= 0 || n <= 0 || (n % 16) != 0) return MOTE_ERR_SHAPE;
+  if (m >= (int64_t(1) << 38) / n) return MOTE_ERR_SHAPE;
+  if (!aligned16(W) || !aligned16(packed) || !aligned16(ws)) return MOTE_ERR_ALIGN;
+  if (ws_bytes < mote_ternarize_workspace_bytes()) return MOTE_ERR_WORKSPACE;
+  return ternarize_with_bins(W, w_dtype, m * n, packed, alpha, static_cast<unsigned long long*>(ws),
+                             static_cast<cudaStream_t>(stream_));
+}
+
 // ---------------------------------------------------------------------------------------------
 // mote_ternarize_pack_static: the same quantizer for callers that have no scratch buffer to give.
 // The exponent bins live in a device array that is part of the loaded library image.
@@ -192,7 +202,6 @@ namespace mote {
 // 256 bins x 8 bytes.  One copy per GPU that loads the library, held until the process exits.
 static __device__ __align__(256) unsigned long long g_static_bins[kBins];
 
-constexpr int kMaxDevices = 64;
 static unsigned long long* g_static_bins_ptr[kMaxDevices];   // device address of g_static_bins, per device
 static std::mutex g_static_bins_mutex;
 
@@ -225,25 +234,5 @@ extern "C" mote_status_t mote_ternarize_pack_static(const void* W, int w_dtype, 
   unsigned long long* bins = nullptr;
   const mote_status_t st = static_bins_address(&bins);
   if (st != MOTE_OK) return st;
-  cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-  const int64_t total = m * n;
-  const int64_t n_vec = total / 4, n_words = total / 16;
-  // the array still holds the previous call's sums
-  MOTE_CUDA_OK(cudaMemsetAsync(bins, 0, kBins * sizeof(unsigned long long), stream));
-  const int threads = 256;
-  const int blocks_a = (int)std::min<int64_t>((n_vec + threads - 1) / threads, 148 * 8);
-  const int blocks_c = (int)std::min<int64_t>((n_words + threads - 1) / threads, 148 * 16);
-  if (w_dtype == MOTE_DTYPE_BF16)
-    abs_sum_bins_kernel<true><<<blocks_a, threads, 0, stream>>>(W, n_vec, bins);
-  else
-    abs_sum_bins_kernel<false><<<blocks_a, threads, 0, stream>>>(W, n_vec, bins);
-  MOTE_LAUNCH_OK();
-  alpha_finalize_kernel<<<1, 32, 0, stream>>>(bins, (double)total, alpha);
-  MOTE_LAUNCH_OK();
-  if (w_dtype == MOTE_DTYPE_BF16)
-    pack_codes_kernel<true><<<blocks_c, threads, 0, stream>>>(W, n_words, alpha, reinterpret_cast<uint32_t*>(packed));
-  else
-    pack_codes_kernel<false><<<blocks_c, threads, 0, stream>>>(W, n_words, alpha, reinterpret_cast<uint32_t*>(packed));
-  MOTE_LAUNCH_OK();
-  return MOTE_OK;
+  return ternarize_with_bins(W, w_dtype, m * n, packed, alpha, bins, static_cast<cudaStream_t>(stream_));
 }

@@ -132,6 +132,19 @@ __device__ __forceinline__ int item_k_range(const UmmaArgs& a, int item, int& kb
   return split;
 }
 
+// What a CTA does after one of its bounded waits has run out (abort flag raised in shared memory):
+// give copies and MMAs still in flight time to land before shared memory and TMEM go away ...
+__device__ __forceinline__ void drain_after_abort(volatile int* abort_flag) {
+  if (*abort_flag) {
+    const uint64_t t0 = globaltimer_ns();
+    while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
+  }
+}
+// ... and raise the device status word the host reads with mote_device_status.
+__device__ __forceinline__ void report_abort(volatile int* abort_flag, uint32_t* status) {
+  if (*abort_flag) atomicExch(status, 1u);
+}
+
 // ------------------------------------------------------------------------------------------------
 template <int MODE>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -569,11 +582,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
   }
 
   // ------------------------------------------------------------------ teardown
-  if (*abort_flag) {
-    // give copies and MMAs still in flight time to land before shared memory and TMEM go away
-    const uint64_t t0 = globaltimer_ns();
-    while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
-  }
+  drain_after_abort(abort_flag);
   tc_fence_before();
   __syncthreads();
   if (warp == 2) {
@@ -581,7 +590,33 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
     tc_fence_after();
     tmem_dealloc(tmem_base, kTmemCols);
   }
-  if (threadIdx.x == 0 && *abort_flag) atomicExch(a.status, 1u);
+  if (threadIdx.x == 0) report_abort(abort_flag, a.status);
+}
+
+// One CTA that runs the GEMM kernels' bounded wait to its limit: an mbarrier nothing ever arrives
+// at, no copy and no MMA in flight.  The wait gives up after limit_ns, the CTA takes the same
+// teardown as the GEMM (drain, status word) and returns normally; the context stays usable.
+__global__ void bounded_wait_selftest_kernel(uint32_t* status, uint64_t limit_ns) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_word;
+  volatile int* abort_flag = &abort_word;
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&bar), 1);
+    abort_word = 0;
+    fence_barrier_init();
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) (void)mbar_wait(smem_u32(&bar), 0, abort_flag, limit_ns);
+  __syncthreads();
+  drain_after_abort(abort_flag);
+  __syncthreads();
+  if (threadIdx.x == 0) report_abort(abort_flag, status);
+}
+
+mote_status_t launch_bounded_wait_selftest(uint32_t* status, uint64_t limit_ns, cudaStream_t stream) {
+  bounded_wait_selftest_kernel<<<1, 32, 0, stream>>>(status, limit_ns);
+  MOTE_LAUNCH_OK();
+  return MOTE_OK;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -629,14 +664,9 @@ template <int MODE>
 static mote_status_t launch_umma(const CUtensorMap& ta, const CUtensorMap& tb0, const CUtensorMap& tb1,
                                  const UmmaArgs& a, int max_items, cudaStream_t stream, bool pdl) {
   using TR = ModeTraits<MODE>;
-  static bool attr_set = false;
-  if (!attr_set) {
-    MOTE_CUDA_OK(cudaFuncSetAttribute(umma_gemm_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TR::kSmem));
-    attr_set = true;
-  }
-  int dev = 0, sms = 148;
-  MOTE_CUDA_OK(cudaGetDevice(&dev));
-  MOTE_CUDA_OK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+  static PerDeviceOnce attr_once;                  // one per MODE (this function is a template)
+  MOTE_CUDA_OK(set_max_dynamic_smem(attr_once, umma_gemm_kernel<MODE>, (int)TR::kSmem));
+  const int sms = device_sm_count();
   const int grid = std::max(1, std::min(sms, max_items));
   if (pdl) MOTE_CUDA_OK(launch_pdl(umma_gemm_kernel<MODE>, dim3(grid), dim3(kThreads), TR::kSmem, stream, ta, tb0, tb1, a));
   else umma_gemm_kernel<MODE><<<grid, kThreads, TR::kSmem, stream>>>(ta, tb0, tb1, a);
@@ -654,8 +684,7 @@ mote_status_t launch_ternary_umma(const TernaryGemmArgs& g, bool gateup, const i
   // a down projection with few row tiles: 128-wide tiles double the items (the weights are the
   // traffic here, and they are read once either way)
   if (!gateup && bn > 128) {
-    int dev = 0, sms = 148;
-    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int sms = device_sm_count();
     if (max_mtiles * (g.N / bn) * 2 <= sms) bn = 128;
   }
   if (!make_map_2d(&ta, g.qa, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, (uint64_t)g.P, (uint64_t)g.K, 128, 128,
@@ -690,12 +719,7 @@ mote_status_t launch_ternary_umma(const TernaryGemmArgs& g, bool gateup, const i
 // occupy the SMs (one row tile of c3: 6 tiles for 27 MB of weights), so each tile's K range is cut
 // into up to 16 items whose partial sums the caller adds.  At most 4096 partial rows in all.
 int shared_down_k_splits(int64_t T, int N, int K) {
-  static int sms = 0;
-  if (sms == 0) {
-    int dev = 0, v = 148;
-    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev);
-    sms = v;
-  }
+  const int sms = device_sm_count();
   const int64_t n_tiles = ((T + 127) / 128) * (N / pick_bn(N));
   if (n_tiles * 2 > sms) return 1;
   int64_t splits = std::min<int64_t>(16, sms / n_tiles);

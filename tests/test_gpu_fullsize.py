@@ -83,3 +83,18 @@ def test_paper_3b_layer_rtn_shared_expert_decode_and_prefill(mote, bits):
     for T in (1, 160):
         rep = check_forward(mote, layer_gpu, layer_or, synth.tokens(wl.with_T(T)))
         assert rep["rel_fro"] < 5e-3
+
+
+@pytest.mark.parametrize("T", [1, 32])
+def test_c5_shape_decode_layer(mote, T):
+    # one layer of the c5 stack at its own shape (d2048 f11008, 16 routed experts, top-2, bf16 shared
+    # expert), host-drawn weights, automatic path (the weight stream at these batch sizes), every tap
+    wl = synth.WORKLOADS["c5"].with_T(T)
+    master = synth.master_layer(wl, layer=0)
+    layer_or = O.build_layer(master)
+    layer_gpu = mote.MoteLayer.from_master(master)
+    check_packed_layer(layer_gpu, layer_or)
+    del master
+    rep = check_forward(mote, layer_gpu, layer_or, synth.tokens(wl))
+    assert rep["tokens"] == T and rep["counts"].sum() == 2 * T
+    assert rep["rel_fro"] < 5e-3

@@ -8,7 +8,7 @@ import torch
 
 from oracle import mote_oracle as O
 from workloads import synth
-from parity_utils import REL_FRO_TOL, bf16_bits, bf16_tensor
+from parity_utils import REL_FRO_TOL, assert_elementwise_close, assert_valid_near_tie_pick, bf16_bits, bf16_tensor
 
 pytestmark = pytest.mark.gpu
 
@@ -134,3 +134,42 @@ def test_stack_forward_can_be_captured_in_a_cuda_graph(mote, T):
     graph.replay()
     torch.cuda.synchronize()
     assert torch.equal(out, want2)
+
+
+def test_c5_shape_stack_per_layer_parity_on_the_gpus_own_inputs(mote):
+    """Three layers of the c5 stack at its own shape (d2048 f11008 E16 k2, bf16 shared expert),
+    host-drawn weights, a decode batch of 32: every layer is compared with the oracle on the
+    residual stream the GPU itself produced for it (stands for layers sampled from the 36-layer
+    stack: every layer has the same shape and its own seeded weights)."""
+    n_layers, T = 3, 32
+    wl = synth.WORKLOADS["c5"].with_T(T)
+    layers, oracles = [], []
+    for l in range(n_layers):
+        master = synth.master_layer(wl, layer=l)
+        layers.append(mote.MoteLayer.from_master(master))
+        oracles.append(O.build_layer(master))
+        del master
+    stack = mote.MoteStack(layers)
+    x = bf16_tensor(synth.tokens(wl))
+    taps = torch.zeros((n_layers, T, wl.d), dtype=torch.bfloat16, device="cuda")
+    out = mote.mote_stack_forward(stack, x, layer_inputs=taps)
+    torch.cuda.synchronize()
+    assert mote.lib.mote_device_status(stack._ws.data_ptr(), None) == 0
+    assert torch.equal(taps[0], x)
+    for l in range(n_layers):
+        res = taps[l].contiguous()
+        xin = mote.mote_rms_norm(res, 1e-6)
+        got_t = taps[l + 1] if l + 1 < n_layers else out
+        # the stack's layer equals a stand-alone call on the same input, bit for bit
+        idx_taps = layers[l].alloc_taps(T, names=["topk_idx"])
+        alone = mote.mote_moe_forward(layers[l], xin, residual=res, taps=idx_taps)
+        assert torch.equal(alone, got_t), l
+        ref = O.moe_forward(oracles[l], bf16_bits(xin), residual_bf16=bf16_bits(res),
+                            near_tie_choice=idx_taps["topk_idx"].cpu().numpy())
+        for t in np.nonzero(ref["near_tie"])[0]:
+            assert_valid_near_tie_pick(idx_taps["topk_idx"][t].cpu().numpy(), ref["logits"][t], wl.k)
+        assert np.array_equal(idx_taps["topk_idx"].cpu().numpy(), ref["topk_idx"])
+        got = O.bf16_to_f32(bf16_bits(got_t)).astype(np.float64)
+        err = np.linalg.norm(got - ref["out"]) / np.linalg.norm(ref["out"])
+        assert err <= REL_FRO_TOL, (l, err)
+        assert_elementwise_close(got, ref["out"], f"layer {l}")

@@ -230,3 +230,60 @@ def test_rtn_shared_ffn_brute_force_and_error_scale(bits):
     plain = O.shared_ffn(x, layer["sh_gate"], layer["sh_up"], layer["sh_down"])
     rel = np.linalg.norm(got - plain) / np.linalg.norm(plain)
     assert rel < (0.05 if bits == 8 else 0.6)
+
+
+# ------------------------------------------------------------------ Eq. 3-4 with an imposed selection
+@pytest.mark.parametrize("norm_topk", [1, 0])
+def test_near_tie_choice_takes_the_other_valid_pick_and_recomputes_the_gate(norm_topk):
+    """A token whose k-th and (k+1)-th logits tie exactly may be routed either way by an fp32
+    router.  moe_forward(near_tie_choice=...) must take the imposed selection for that token only,
+    give it the gate weights of Eq. 3 (softmax over the selected k, or over all E experts) from
+    the oracle's own logits, and leave every other token alone."""
+    d, f, E, k, T = 16, 32, 4, 2, 3
+    wl = synth.custom("tie", d, f, E, k, T, 31, norm_topk=norm_topk)
+    master = synth.master_layer(wl)
+    # hand-made router: token 0 has logits (2, 1, 1, -1): experts 1 and 2 tie for the second slot
+    Wr = np.zeros((E, d), np.float32)
+    Wr[0, 0], Wr[1, 0], Wr[2, 0], Wr[3, 0] = 2.0, 1.0, 1.0, -1.0
+    Wr[:, 1] = [0.5, -0.25, 3.0, 0.125]                 # tokens 1, 2 use channel 1: no tie
+    master["Wr"], master["router_bias"] = Wr, None
+    layer = O.build_layer(master)
+    xf = np.zeros((T, d), np.float32)
+    xf[0, 0] = 1.0
+    xf[1, 1] = 1.0
+    xf[2, 1] = -2.0
+    xf[:, 2:] = np.random.default_rng(5).standard_normal((T, d - 2)).astype(np.float32)
+    x = _bf16(xf)
+    base = O.moe_forward(layer, x)
+    assert base["near_tie"].tolist() == [True, False, False]
+    assert base["topk_idx"][0].tolist() == [0, 1]        # ties go to the lower index
+    # the other valid pick for token 0; nonsense for the unflagged tokens, which must be ignored
+    choice = np.array([[0, 2], [3, 3], [1, 1]], np.int32)
+    got = O.moe_forward(layer, x, near_tie_choice=choice)
+    assert got["topk_idx"][0].tolist() == [0, 2]
+    assert np.array_equal(got["topk_idx"][1:], base["topk_idx"][1:])
+    assert np.array_equal(got["topk_w"][1:], base["topk_w"][1:])
+    assert np.array_equal(got["out"][1:], base["out"][1:])
+    # gate weights of token 0 by scalar arithmetic on the exact logits (2, 1, 1, -1)
+    lg = [2.0, 1.0, 1.0, -1.0]
+    sel = [0, 2]
+    den = sum(math.exp(lg[e]) for e in (sel if norm_topk else range(E)))
+    want = [math.exp(lg[e]) / den for e in sel]
+    assert np.allclose(got["topk_w"][0], want, rtol=1e-12)
+    assert np.allclose(got["topk_w"][0], base["topk_w"][0], rtol=1e-12)   # equal logits, equal weights
+    if norm_topk:
+        assert abs(got["topk_w"][0].sum() - 1.0) < 1e-12
+    else:
+        assert got["topk_w"][0].sum() < 0.9              # the mass of the unselected experts is missing
+    # dispatch follows the imposed selection, and the output is the sum over the imposed experts:
+    # recompute token 0 from the per-expert stages
+    assert np.array_equal(np.diff(got["offsets"]), np.bincount(got["topk_idx"].ravel(), minlength=E))
+    qx, bx, _ = O.quant_act(x[:1])
+    total = O.shared_ffn(x[:1], layer["sh_gate"], layer["sh_up"], layer["sh_down"])[0]
+    for j, e in enumerate(sel):
+        r = O.ternary_expert(qx, bx, layer["codes_gate"][e], layer["alpha_gate"][e], layer["codes_up"][e],
+                             layer["alpha_up"][e], layer["codes_down"][e], layer["alpha_down"][e])
+        total = total + want[j] * r["y"][0]
+    assert np.allclose(got["out"][0], total, rtol=1e-12, atol=1e-15)
+    # experts 1 and 2 hold different weights, so the imposed pick really changes the result
+    assert not np.allclose(got["out"][0], base["out"][0], rtol=1e-6)

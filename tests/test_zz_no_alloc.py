@@ -11,6 +11,8 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import mote_oracle as O
+
 
 @pytest.fixture(scope="module")
 def mote():
@@ -25,19 +27,28 @@ def _w(shape, seed, scale, dtype=torch.float32):
 @pytest.mark.gpu
 def test_static_scratch_matches_workspace_entry_point_twice_in_a_row(mote):
     cases = [_w((512, 1024), 41, 0.02), _w((96, 320), 42, 3.0), _w((256, 512), 43, 0.02, torch.bfloat16)]
-    for W in cases:
+    for i, W in enumerate(cases):
         m, n = W.shape
         want_packed, want_alpha = mote.mote_ternarize_pack(W)
         packed = torch.full((m, n // 4), 0xFF, dtype=torch.uint8, device="cuda")
         alpha = torch.full((1,), -1.0, dtype=torch.float32, device="cuda")
         torch.cuda.synchronize()
         before = torch.cuda.memory_allocated()
+        free_before = torch.cuda.mem_get_info()[0]
         mote.mote_ternarize_pack_static(W, packed, alpha)
         torch.cuda.synchronize()
         assert torch.cuda.memory_allocated() == before
+        # the driver's view too, which would also see an allocation made inside the library (from the
+        # second call on: the first use of a library on a device may load its code there)
+        if i > 0:
+            assert torch.cuda.mem_get_info()[0] >= free_before
         # integer and byte work: bit-exact, as everywhere else in the suite
         assert alpha.item() == want_alpha.item()
         assert torch.equal(packed, want_packed)
+        # and against the oracle directly (Eq. 7, 9), not only through the other entry point
+        codes, a = O.ternarize(W.float().cpu().numpy())
+        assert alpha.item() == float(a)
+        assert np.array_equal(packed.cpu().numpy(), O.pack_codes(codes))
 
 
 def test_static_scratch_rejects_oversize_and_bad_arguments(mote):
