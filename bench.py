@@ -1,22 +1,30 @@
 #!/usr/bin/env python
 """Benchmark of the MoTE FFN-layer forward pass on B200.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2|c4|c3-T|c1] [--impl ours|reference]
-                  [--shared-bits 16|8|4]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c4|c2|c1|c3-T|c5-T|p3-T ...]
+                  [--impl ours|reference] [--shared-bits 16|8|4] [--no-sweep]
 
 One "step" is one pass of the whole layer (route, dispatch, Q_a(x), gate/up ternary GEMM, Q_a(h),
-down ternary GEMM, shared bf16 FFN, combine) over one batch of synthetic tokens.  Weights are
-ternarized once, before the timed region (offline step).  Prints ONE JSON line.
+down ternary GEMM, shared bf16 FFN, combine) over one batch of synthetic tokens; for the stacked
+workloads (c5, p*) one pass of all their layers.  Weights are ternarized once, before the timed
+region (offline step).  Prints ONE JSON line.
+
+The headline record is the workload named by --workload (default c4, the largest single layer);
+K steps are timed exactly.  At one GPU the line also carries "workloads": a compact record of every
+workload of the five configurations (c1, c2, c3 at 1/8/32/64 tokens, c4, c5 at 1/32/2048 tokens),
+each timed for about a second.
 
 Multi-GPU: the layer is token-parallel with no exchange step, so every rank holds a full replica
 and its own batch (weak scaling, no collective on the data path); the job value is the sum of the
-ranks' tokens over the slowest rank's time.
+ranks' tokens over the slowest rank's time.  `--gpus N` without a launcher (no WORLD_SIZE in the
+environment) starts the N replica processes itself.
 """
 from __future__ import annotations
 
 import argparse
 import json
 import os
+import socket
 import statistics
 import subprocess
 import sys
@@ -32,16 +40,20 @@ sys.path.insert(0, ROOT)
 from workloads import synth  # noqa: E402
 
 L2_FLUSH_BYTES = 512 << 20
-NOMINAL_INT8_OVER_BF16 = 2.0      # dense tensor peak ratio int8 : bf16 (4.5 vs 2.25 POP/s nominal)
+NOMINAL = {"int8_tops": 4500.0, "bf16_tflops": 2250.0, "hbm_gbs": 8000.0}     # datasheet, dense
+SWEEP = ["c1", "c2", "c3-1", "c3-8", "c3-32", "c3-64", "c4", "c5-1", "c5-32", "c5-2048"]
+SUSTAINED_MIN_MS = 300.0          # a timed region at least this long is compared with sustained peaks
 
 
 def parse_workload(name: str) -> synth.Workload:
-    if name.startswith("c3-"):
-        return synth.WORKLOADS["c3"].with_T(int(name[3:]))
-    if "-" in name:                                     # stacked workloads: c5-32, p3-1, p05-2048 ...
+    if "-" in name:                                     # c3-8, c5-32, p3-1, p05-2048 ...
         base, T = name.split("-", 1)
         return synth.WORKLOADS[base].with_T(int(T))
     return synth.WORKLOADS[name]
+
+
+def workload_label(wl: synth.Workload) -> str:
+    return wl.name if wl.T == synth.WORKLOADS[wl.name].T and wl.name not in ("c3", "c5") else f"{wl.name}-{wl.T}"
 
 
 def measured_peaks():
@@ -70,6 +82,7 @@ class ClockSampler:
             self.thread.start()
         except OSError:
             self.proc = None
+        return self
 
     def _read(self):
         for line in self.proc.stdout:
@@ -98,12 +111,6 @@ class ClockSampler:
                 "samples": len(sm)}
 
 
-# ncu dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the captures
-# summarised under profiles/ (null once the kernel has changed since, or where no capture exists)
-NCU_TRAFFIC_BYTES = {("c2", "gateup_ternary"): 42.88e6, ("c4", "gateup_ternary"): 610.09e6,
-                     ("c3-1", "gateup_ternary"): 69.92e6}
-
-
 def stage_work(wl: synth.Workload, stage: str, stream_path: bool, experts_touched: float, shared_bits: int = 16,
                peaks: dict | None = None):
     """Algorithmic work of one launch of a stage: (amount, kind), kind 'int8' | 'bf16' | 'bytes'.
@@ -126,7 +133,7 @@ def stage_work(wl: synth.Workload, stage: str, stream_path: bool, experts_touche
     if stage in gemm:
         ops, kind, nbytes = gemm[stage]
         if peaks is not None:
-            t_ops = ops / (peaks["bf16_tflops"] * 1e12 * (NOMINAL_INT8_OVER_BF16 if kind == "int8" else 1.0))
+            t_ops = ops / ((peaks["int8_tops"] if kind == "int8" else peaks["bf16_tflops"]) * 1e12)
             if nbytes / (peaks["hbm_gbs"] * 1e9) > t_ops:
                 return nbytes, "bytes"
         return ops, kind
@@ -157,66 +164,89 @@ def job_tokens_per_s(world: int, tokens_per_rank: int, steps: int, total_ms: flo
     return world * tokens_per_rank * steps / (total_ms * 1e-3)
 
 
-def run_ours(args):
-    rank = int(os.environ.get("RANK", 0))
-    local_rank = int(os.environ.get("LOCAL_RANK", 0))
-    world = int(os.environ.get("WORLD_SIZE", 1))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback for the product path")
-    torch.cuda.set_device(local_rank)
-    dev = torch.device("cuda", local_rank)
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=dev)
-    wl = parse_workload(args.workload)
-    import paper_2506_14435_b200 as mote
-    from paper_2506_14435_b200.binding import mote_moe_forward_host, mote_moe_forward_profile
+def replica_command(n: int, argv: list[str], port: int) -> list[str]:
+    """The launch of n replica processes of this script on one node (what `--gpus n` runs when no
+    launcher has set WORLD_SIZE): one rank per GPU, rendezvous on the loopback address."""
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+            "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__), *argv]
 
-    n_layers = wl.n_layers if args.layers is None else args.layers
-    is_stack = wl.n_layers > 1
-    master = None
+
+def free_port() -> int:
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def int8_peak(mote_binding, rank: int, local_rank: int) -> dict:
+    """The int8 tensor pipe's speed of light, measured with the library's MMA-only kernel
+    (tcgen05.mma.kind::i8 M128 N256 K32 on shared-memory-resident operands): a burst figure (best of
+    a few 5 ms launches from idle clocks) and a sustained one (median launch of the second half of
+    about a second of back-to-back launches, clocks sampled meanwhile)."""
+    burst = mote_binding.mote_int8_mma_peak(800, repeats=5)
+    sampler = ClockSampler(local_rank).start() if rank == 0 else None
+    long = mote_binding.mote_int8_mma_peak(1600, repeats=80)
+    clocks = sampler.stop() if sampler else None
+    ms = long["ms_in_order"][len(long["ms_in_order"]) // 2:]
+    sustained = long["ops"] / (statistics.median(ms) * 1e-3) / 1e12
+    return {"burst_tops": burst["tops_best"], "sustained_tops": sustained, "sustained_clocks": clocks,
+            "how": "libmote mote_int8_mma_peak: tcgen05.mma.kind::i8 M128xN256xK32, smem-resident operands, all SMs"}
+
+
+class LayerSet:
+    """The device-resident layers of one base workload (c3, c5 ... share them across batch sizes)."""
+
+    def __init__(self, base: synth.Workload, mote, dev, n_layers: int | None, shared_bits: int, path: str):
+        self.base, self.mote, self.dev = base, mote, dev
+        self.is_stack = base.n_layers > 1
+        n = base.n_layers if n_layers is None else n_layers
+        self.master = None
+        if self.is_stack:
+            # 36 layers of 0.8 G weights each: drawn on the device (minutes on the host); every layer distinct
+            self.layers = [mote.MoteLayer.from_device_draws(base.d, base.f, base.E, base.k, base.norm_topk,
+                                                            synth.device_draw(base, l, dev), device=dev) for l in range(n)]
+        else:
+            self.master = synth.master_layer(base)
+            self.layers = [mote.MoteLayer.from_master(self.master, device=dev)]
+        if shared_bits != 16:                               # offline step: RTN codes of the shared expert
+            self.layers = [l.quantize_shared(shared_bits) for l in self.layers]
+            torch.cuda.empty_cache()
+        if path != "auto":                                  # force one implementation (default: the library picks)
+            for l in self.layers:
+                l.path = {"simt": mote.PATH_SIMT, "tensor": mote.PATH_TENSOR, "stream": mote.PATH_STREAM}[path]
+        self.stack = mote.MoteStack(self.layers) if self.is_stack else None
+
+
+def measure(ls: LayerSet, wl: synth.Workload, args, steps: int | None, rank: int, local_rank: int, world: int,
+            peaks: dict, flush: torch.Tensor) -> dict:
+    """Times one workload: `steps` steps exactly (or, steps=None, as many as fill about a second)
+    device-resident, then the per-stage times of the same launch configuration over a loop of
+    similar length, then the end-to-end loop with host buffers."""
+    mote, dev, layers, is_stack = ls.mote, ls.dev, ls.layers, ls.is_stack
+    from paper_2506_14435_b200.binding import mote_moe_forward_host, mote_moe_forward_profile
     if is_stack:
-        # 36 layers of 0.8 G weights each: drawn on the device (minutes on the host); every layer distinct
-        layers = [mote.MoteLayer.from_device_draws(wl.d, wl.f, wl.E, wl.k, wl.norm_topk,
-                                                   synth.device_draw(wl, l, dev), device=dev) for l in range(n_layers)]
-        stack = mote.MoteStack(layers)
         x = synth.device_tokens(wl, dev, stream=rank)
         x_host = x.cpu().pin_memory()
-        x_bits = None
     else:
-        master = synth.master_layer(wl)
-        layers = [mote.MoteLayer.from_master(master, device=dev)]
         x_bits = synth.tokens(wl, stream=rank)
         x_host = torch.from_numpy(x_bits.view(np.int16).copy()).view(torch.bfloat16).pin_memory()
         x = x_host.to(dev)
-    if args.shared_bits != 16:                          # offline step: RTN codes of the shared expert
-        layers = [l.quantize_shared(args.shared_bits) for l in layers]
-        if is_stack:
-            stack = mote.MoteStack(layers)
-        torch.cuda.empty_cache()
     out_host = torch.empty_like(x_host).pin_memory()
     out = torch.empty_like(x)
-    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
     stream = torch.cuda.current_stream()
-    if args.path != "auto":                             # force one implementation (default: the library picks)
-        for l in layers:
-            l.path = {"simt": mote.PATH_SIMT, "tensor": mote.PATH_TENSOR, "stream": mote.PATH_STREAM}[args.path]
-        if is_stack:
-            stack = mote.MoteStack(layers)
     tensor_ok = wl.d % 128 == 0 and wl.f % 128 == 0     # the library's own choice, restated for the work model
     stream_path = (wl.T <= (32 if tensor_ok else 64) and wl.d % 64 == 0 and wl.f % 64 == 0) \
         if args.path == "auto" else args.path == "stream"
 
     def step_device():
         if is_stack:
-            mote.mote_stack_forward(stack, x, out=out)
+            mote.mote_stack_forward(ls.stack, x, out=out)
         else:
             mote.mote_moe_forward(layers[0], x, out=out)
 
     def step_host():
         if is_stack:                                    # host buffers in and out around the C-ABI call
             x.copy_(x_host, non_blocking=True)
-            mote.mote_stack_forward(stack, x, out=out)
+            mote.mote_stack_forward(ls.stack, x, out=out)
             out_host.copy_(out, non_blocking=True)
             torch.cuda.synchronize()
         else:
@@ -254,6 +284,9 @@ def run_ours(args):
     for _ in range(args.warmup):
         step_device()
     launches_per_step = mote.lib.mote_last_launch_count()
+    if steps is None:                                   # fill about a second
+        est = statistics.median(timed_loop(step_device, 3))
+        steps = int(min(2000, max(10, 1000.0 / max(est + 0.25, 1e-3))))
     step_timed = step_device
     if args.graph:
         # the whole step (every launch of the C-ABI call) captured once in a CUDA graph and replayed:
@@ -271,18 +304,19 @@ def run_ours(args):
         for _ in range(3):
             step_timed()
     barrier()
-    sampler = ClockSampler(local_rank)
-    if rank == 0:
-        sampler.start()
-    per_step = timed_loop(step_timed, args.steps)
+    sampler = ClockSampler(local_rank).start() if rank == 0 else None
+    per_step = timed_loop(step_timed, steps)
     barrier()
+    clocks = sampler.stop() if sampler else None
     total_ms = sum(per_step)
 
-    # ---- per-stage device times of the same launch configuration (events on the launch stream)
+    # ---- per-stage device times of the same launch configuration (events on the launch stream), over a
+    # loop about as long as the timed one, so that both run at the same clocks
     stage_acc = {}
-    n_prof = max(3, min(args.steps, 10))
+    n_prof = max(3, min(steps, int(500.0 / max(total_ms / steps, 1e-3)) + 1))
+    sampler = ClockSampler(local_rank).start() if rank == 0 else None
     for i in range(n_prof):
-        flush.fill_(i)
+        flush.fill_(i & 0xFF)
         cur = x
         tot = {}
         for layer in layers:
@@ -294,7 +328,7 @@ def run_ours(args):
             cur = nxt
         for k_, v in tot.items():
             stage_acc.setdefault(k_, []).append(v)
-    clocks = sampler.stop() if rank == 0 else None
+    stage_clocks = sampler.stop() if sampler else None
     stage_ms = {k_: statistics.mean(v) for k_, v in stage_acc.items()}     # summed over the layers
 
     # ---- end to end: host buffers in and out
@@ -302,7 +336,7 @@ def run_ours(args):
         step_host()
     barrier()
     e2e_ms = []
-    for i in range(args.steps):
+    for i in range(steps):
         flush.fill_(i & 0xFF)
         torch.cuda.synchronize()
         t0 = time.perf_counter()
@@ -310,64 +344,171 @@ def run_ours(args):
         e2e_ms.append((time.perf_counter() - t0) * 1e3)
     barrier()
     e2e_total = sum(e2e_ms)
+    if not bool(torch.isfinite(out.float()).all()):
+        raise SystemExit("non-finite layer output: the timing would not be valid")
 
     total_ms, e2e_total = max_over_ranks([total_ms, e2e_total], dev, world)
+    ms_per_step = total_ms / steps
+    sustained = total_ms >= SUSTAINED_MIN_MS
+    n_l = len(layers)
+    dom = max(stage_ms, key=stage_ms.get)
+    work, kind = stage_work(wl, dom, stream_path, experts_touched, args.shared_bits, peaks)
+    dur_s = stage_ms[dom] * 1e-3 / n_l                  # average duration of one launch of that kernel
+    from paper_2506_14435_b200 import traffic
+    label = workload_label(wl)
+    if kind == "bytes":
+        roof = dict(bound="hbm", achieved=work / dur_s / 1e9, peak=peaks["hbm_gbs"], unit="GB/s",
+                    peak_source=f"of {peaks['source']} (copy bandwidth)", frac_of_nominal=work / dur_s / 1e9 / NOMINAL["hbm_gbs"])
+    elif kind == "int8":
+        peak = peaks["int8_tops_sustained"] if sustained else peaks["int8_tops"]
+        roof = dict(bound="tensor", achieved=work / dur_s / 1e12, peak=peak, unit="TOP/s",
+                    peak_source=("of measured: the library's tcgen05 kind::i8 MMA-only loop, " +
+                                 ("sustained figure (timed region of %.0f ms)" % total_ms if sustained else "burst figure")),
+                    peak_burst=peaks["int8_tops"], peak_sustained=peaks["int8_tops_sustained"],
+                    peak_2x_bf16_burst=2.0 * peaks["bf16_tflops"], frac_of_nominal=work / dur_s / 1e12 / NOMINAL["int8_tops"])
+    else:
+        peak = peaks["bf16_tflops_sustained"] if sustained else peaks["bf16_tflops"]
+        roof = dict(bound="tensor", achieved=work / dur_s / 1e12, peak=peak, unit="TFLOP/s",
+                    peak_source=f"of {peaks['source']} (cuBLAS bf16, " + ("sustained)" if sustained else "burst)"),
+                    frac_of_nominal=work / dur_s / 1e12 / NOMINAL["bf16_tflops"])
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    roof["traffic"] = traffic.lookup(label, dom, "stream" if stream_path else "tensor")
+    roof["kernel"] = dom
+    roof["kernel_ms"] = dur_s * 1e3
+    roof["algorithmic_work_per_launch"] = work
+    roof["sm_mhz"] = stage_clocks["sm_mhz"] if stage_clocks else None
+    weight_bytes = n_l * (experts_touched * 3 * wl.d * wl.f / 4 + 3.0 * wl.d * wl.f * args.shared_bits / 8)
+    sm_mhz = clocks["sm_mhz"] if clocks else None
+    rec = {
+        "workload": label, "wl": wl, "steps": steps, "ms_per_step": ms_per_step, "total_ms": total_ms,
+        "us_per_layer": ms_per_step * 1e3 / n_l, "us_per_token": ms_per_step * 1e3 / wl.T,
+        "tokens_per_s": job_tokens_per_s(world, wl.T, steps, total_ms),
+        "ms_x_sm_mhz": ms_per_step * sm_mhz if sm_mhz else None,
+        "layers": n_l, "experts_touched": experts_touched, "stream_path": stream_path,
+        "stage_ms": stage_ms, "roofline": roof,
+        "weights_touched_gbs": weight_bytes / (ms_per_step * 1e-3) / 1e9,
+        "e2e": {"value": job_tokens_per_s(world, wl.T, steps, e2e_total), "unit": "tokens/s",
+                "h2d_bytes_per_step": int(x_host.numel() * 2), "d2h_bytes_per_step": int(out_host.numel() * 2)},
+        "gpu_launches": launches_per_step * steps, "launches_per_step": launches_per_step, "clocks": clocks,
+    }
+    # the two quantities the targets are stated on
+    P = wl.T * wl.k
+    if stream_path:
+        rec["decode_hbm"] = {"weight_bytes_per_step": weight_bytes, "gbs": rec["weights_touched_gbs"],
+                             "frac_of_measured": rec["weights_touched_gbs"] / peaks["hbm_gbs"],
+                             "frac_of_nominal": rec["weights_touched_gbs"] / NOMINAL["hbm_gbs"],
+                             "note": "all weight bytes touched (2-bit codes of the experts that received tokens + the "
+                                     "shared expert) over the whole step; the stream kernels cover both"}
+    else:
+        t_routed = (stage_ms["gateup_ternary"] + stage_ms["down_ternary"]) * 1e-3 / n_l
+        t_with_q = t_routed + stage_ms["quant_h"] * 1e-3 / n_l
+        ops = 6.0 * wl.d * wl.f * P
+        pk = peaks["int8_tops_sustained"] if sustained else peaks["int8_tops"]
+        rec["routed_gemms"] = {"int8_ops": ops, "ms": t_routed * 1e3, "tops": ops / t_routed / 1e12,
+                               "frac_of_measured": ops / t_routed / 1e12 / pk,
+                               "frac_of_nominal": ops / t_routed / 1e12 / NOMINAL["int8_tops"],
+                               "frac_of_measured_with_quant_h": ops / t_with_q / 1e12 / pk}
+    return rec
+
+
+def compact(rec: dict) -> dict:
+    r = rec["roofline"]
+    out = {"workload": rec["workload"], "T": rec["wl"].T, "layers": rec["layers"], "steps": rec["steps"],
+           "path": "stream" if rec["stream_path"] else "tensor",
+           "ms_per_step": round(rec["ms_per_step"], 5), "us_per_layer": round(rec["us_per_layer"], 2),
+           "tokens_per_s": round(rec["tokens_per_s"], 1), "ms_x_sm_mhz": rec["ms_x_sm_mhz"],
+           "sm_mhz": rec["clocks"]["sm_mhz"] if rec["clocks"] else None,
+           "dominant": r["kernel"],
+           "roofline": {k: r[k] for k in ("bound", "achieved", "peak", "unit", "frac", "frac_of_nominal", "kernel_ms",
+                                          "algorithmic_work_per_launch", "traffic")},
+           "weights_touched_gbs": round(rec["weights_touched_gbs"], 1),
+           "e2e_tokens_per_s": round(rec["e2e"]["value"], 1), "launches_per_step": rec["launches_per_step"]}
+    for k in ("decode_hbm", "routed_gemms"):
+        if k in rec:
+            out[k] = {a: b for a, b in rec[k].items() if a != "note"}
+    return out
+
+
+def run_ours(args):
+    rank = int(os.environ.get("RANK", 0))
+    local_rank = int(os.environ.get("LOCAL_RANK", 0))
+    world = int(os.environ.get("WORLD_SIZE", 1))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU fallback for the product path")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    import paper_2506_14435_b200 as mote
+    from paper_2506_14435_b200 import binding
+
+    peaks = measured_peaks()
+    i8 = int8_peak(binding, rank, local_rank)
+    peaks["int8_tops"], peaks["int8_tops_sustained"] = i8["burst_tops"], i8["sustained_tops"]
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+
+    wl = parse_workload(args.workload)
+    base = synth.WORKLOADS[wl.name]
+    ls = LayerSet(base, mote, dev, args.layers, args.shared_bits, args.path)
+    head = measure(ls, wl, args, args.steps, rank, local_rank, world, peaks, flush)
+
+    records = {head["workload"]: head}
+    sweep = world == 1 and not args.no_sweep and args.shared_bits == 16 and args.path == "auto" and not args.graph \
+        and args.layers is None
+    cb = None
+    if world == 1 and rank == 0:
+        master, x_bits = ls.master, None
+        if ls.is_stack:                                     # the oracle needs host-drawn weights: layer 0, scaled by the depth
+            master = synth.master_layer(wl)
+        x_bits = synth.tokens(wl)
+        cb = cpu_baseline(wl, master, x_bits, budget_s=12.0, shared_bits=args.shared_bits)
+        if ls.is_stack:
+            cb["value"] /= head["layers"]
+            cb["sample"] += f"; one layer timed, value divided by the {head['layers']} layers of the stack"
+        del master
+    if sweep:
+        for name in SWEEP:
+            w = parse_workload(name)
+            if workload_label(w) in records:
+                continue
+            if w.name != ls.base.name:
+                del ls
+                torch.cuda.empty_cache()
+                ls = LayerSet(synth.WORKLOADS[w.name], mote, dev, None, 16, "auto")
+            records[workload_label(w)] = measure(ls, w, args, None, rank, local_rank, world, peaks, flush)
     if rank != 0:
         if world > 1:
             import torch.distributed as dist
             dist.destroy_process_group()
         return
 
-    peaks = measured_peaks()
-    ms_per_step = total_ms / args.steps
-    tokens_per_s = job_tokens_per_s(world, wl.T, args.steps, total_ms)
     decode = wl.T <= 64
-    dom = max(stage_ms, key=stage_ms.get)
-    work, kind = stage_work(wl, dom, stream_path, experts_touched, args.shared_bits, peaks)
-    dur_s = stage_ms[dom] * 1e-3 / len(layers)          # average duration of one launch of that kernel
-    if kind == "bytes":
-        roof = dict(bound="hbm", achieved=work / dur_s / 1e9, peak=peaks["hbm_gbs"], unit="GB/s")
-    else:
-        peak = peaks["bf16_tflops"] * (NOMINAL_INT8_OVER_BF16 if kind == "int8" else 1.0)
-        roof = dict(bound="tensor", achieved=work / dur_s / 1e12, peak=peak, unit="TOP/s" if kind == "int8" else "TFLOP/s")
-    roof["frac"] = roof["achieved"] / roof["peak"]
-    roof["traffic"] = NCU_TRAFFIC_BYTES.get((wl.name if not decode else f"{wl.name}-{wl.T}", dom))
-    roof["kernel"] = dom
-    roof["kernel_ms"] = dur_s * 1e3
-    roof["algorithmic_work_per_launch"] = work
-    roof["peak_source"] = ("of measured" if peaks["source"] == "measured" else "of fallback") + \
-        (" (bf16 burst x2 nominal int8:bf16 ratio)" if kind == "int8" else "")
-    weight_bytes = len(layers) * (experts_touched * 3 * wl.d * wl.f / 4 + 3.0 * wl.d * wl.f * args.shared_bits / 8)
-    if not bool(torch.isfinite(out.float()).all()):
-        raise SystemExit("non-finite layer output: the timing would not be valid")
     line = {
         "metric": "MoTE layer tokens/sec (prefill)" if not decode else "MoTE layer tokens/sec (decode batch)",
-        "value": tokens_per_s, "unit": "tokens/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": ms_per_step, "us_per_layer": ms_per_step * 1e3 / len(layers),
-        "us_per_token": ms_per_step * 1e3 / wl.T, "higher_is_better": True,
+        "value": head["tokens_per_s"], "unit": "tokens/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": head["ms_per_step"], "us_per_layer": head["us_per_layer"],
+        "us_per_token": head["us_per_token"], "ms_x_sm_mhz": head["ms_x_sm_mhz"], "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "int8xint2->int32 routed, bf16 shared" + (
             "" if args.shared_bits == 16 else f" (weights RTN int{args.shared_bits}, weight-only)"), "data": "synthetic",
-        "config": {"workload": wl.name, "d": wl.d, "f": wl.f, "E": wl.E, "k": wl.k, "T_per_gpu": wl.T,
-                   "layers": len(layers), "experts_touched_per_layer": experts_touched,
+        "config": {"workload": head["workload"], "d": wl.d, "f": wl.f, "E": wl.E, "k": wl.k, "T_per_gpu": wl.T,
+                   "layers": head["layers"], "experts_touched_per_layer": head["experts_touched"],
                    "shared_bits": args.shared_bits, "path": args.path,
                    "launch": "CUDA graph replay of the step" if args.graph else "direct launches",
-                   "pre_norm": "rms, eps 1e-6, unit gain" if is_stack else "none (the caller's)",
+                   "pre_norm": "rms, eps 1e-6, unit gain" if ls.is_stack or wl.n_layers > 1 else "none (the caller's)",
                    "l2": "flushed between timed iterations (512 MiB write)", "parallelism": f"replicas x{world}"},
-        "stage_ms": stage_ms, "roofline": roof,
-        "weights_touched_gbs": weight_bytes / (ms_per_step * 1e-3) / 1e9,
-        "e2e": {"value": job_tokens_per_s(world, wl.T, args.steps, e2e_total), "unit": "tokens/s",
-                "h2d_bytes_per_step": int(x_host.numel() * 2), "d2h_bytes_per_step": int(out_host.numel() * 2)},
-        "gpu_launches": launches_per_step * args.steps, "clocks": clocks,
+        "stage_ms": head["stage_ms"], "roofline": head["roofline"],
+        "weights_touched_gbs": head["weights_touched_gbs"],
+        "e2e": head["e2e"], "gpu_launches": head["gpu_launches"], "clocks": head["clocks"],
+        "int8_peak": i8,
     }
-    if world == 1:
-        if is_stack:                                    # the oracle needs host-drawn weights: layer 0, scaled by the depth
-            master = synth.master_layer(wl)
-            x_bits = synth.tokens(wl)
-        cb = cpu_baseline(wl, master, x_bits, budget_s=12.0, shared_bits=args.shared_bits)
-        if is_stack:
-            cb["value"] /= len(layers)
-            cb["sample"] += f"; one layer timed, value divided by the {len(layers)} layers of the stack"
+    for k in ("decode_hbm", "routed_gemms"):
+        if k in head:
+            line[k] = head[k]
+    if cb is not None:
         line["cpu_baseline"] = cb
+    if sweep:
+        line["workloads"] = [compact(records[workload_label(parse_workload(n))]) for n in SWEEP]
     print(json.dumps(line))
     if world > 1:
         import torch.distributed as dist
@@ -408,6 +549,7 @@ def run_reference(args):
     master = synth.master_layer(wl)
     from oracle import mote_oracle as O
     layer_or = O.build_layer(master)
+    del master
     if args.shared_bits != 16:
         layer_or = O.quantize_shared(layer_or, args.shared_bits)
     x_bits = synth.tokens(wl)
@@ -420,6 +562,8 @@ def run_reference(args):
         O.moe_forward(layer_or, x_bits, token_subset=sub)
     dt = time.perf_counter() - t0
     val = n * args.steps / dt
+    if wl.n_layers > 1:
+        val /= wl.n_layers                                  # one layer timed; a step of the stack is n_layers of them
     decode = wl.T <= 64
     print(json.dumps({
         "impl": "reference",
@@ -427,10 +571,11 @@ def run_reference(args):
         "value": val, "unit": "tokens/s", "n_gpus": int(os.environ.get("WORLD_SIZE", 1)), "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "fp64 / exact integers", "data": "synthetic",
-        "config": {"workload": wl.name, "d": wl.d, "f": wl.f, "E": wl.E, "k": wl.k, "T_per_gpu": wl.T,
-                   "shared_bits": args.shared_bits},
+        "config": {"workload": workload_label(wl), "d": wl.d, "f": wl.f, "E": wl.E, "k": wl.k, "T_per_gpu": wl.T,
+                   "layers": wl.n_layers, "shared_bits": args.shared_bits},
         "cpu_baseline": {"value": val, "unit": "tokens/s", "cores": torch.get_num_threads(), "kind": "oracle",
-                         "sample": f"each step = first {n} of {wl.T} tokens of {wl.name}"},
+                         "sample": f"each step = first {n} of {wl.T} tokens of {wl.name}" +
+                                   (f", one layer (value divided by the {wl.n_layers} layers)" if wl.n_layers > 1 else "")},
         "e2e": {"value": val, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
 
@@ -438,9 +583,10 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=None,
+                    help="timed steps of the headline workload (default: 400 for ours, about a second at c4; 3 for the reference)")
     ap.add_argument("--warmup", type=int, default=3)
-    ap.add_argument("--workload", default="c2")
+    ap.add_argument("--workload", default="c4")
     ap.add_argument("--layers", type=int, default=None, help="layers of a stacked workload (c5-T: default 36)")
     ap.add_argument("--shared-bits", type=int, default=16, choices=[16, 8, 4],
                     help="storage of the shared expert: bf16, or RTN INT8 / INT4 codes (Section 4.3)")
@@ -448,9 +594,17 @@ def main():
                     help="implementation of the layer (auto: the library's own choice per shape)")
     ap.add_argument("--graph", action="store_true",
                     help="time the step as a CUDA graph replay (captured once from the same C-ABI call)")
+    ap.add_argument("--no-sweep", action="store_true", help="leave out the records of the other workloads")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     args = ap.parse_args()
+    if args.steps is None:
+        args.steps = 400 if args.impl == "ours" else 3
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # no launcher: start the replicas ourselves, one process per GPU (the reference arm has one rank's work)
+        if args.impl == "ours" and torch.cuda.device_count() < args.gpus:
+            raise SystemExit(f"--gpus {args.gpus}: only {torch.cuda.device_count()} CUDA device(s) visible")
+        raise SystemExit(subprocess.call(replica_command(args.gpus, sys.argv[1:], free_port())))
     if args.impl == "reference":
         run_reference(args)
     else:

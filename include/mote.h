@@ -332,6 +332,16 @@ mote_status_t mote_device_status(void* ws, void* stream);
  *   limit_ns  1 000 .. 100 000 000 (1 us .. 100 ms); outside -> ERR_SHAPE */
 mote_status_t mote_selftest_bounded_wait(void* ws, uint64_t limit_ns, void* stream);
 
+/* Measurement aid (no counterpart in the paper): the int8 tensor-core speed of light of the device,
+ * as a kernel to be timed by the caller.  One thread block per SM issues n_batches * 64
+ * tcgen05.mma.kind::i8 instructions of the routed expert GEMMs' shape (M128 x N256 x K32,
+ * s8 x u8 -> s32) on operands resident in shared memory: no loads, no unpacking, no epilogue.
+ * Enqueues one kernel on `stream` and writes the number of integer operations it performs
+ * (2 per multiply-accumulate, all SMs) to *ops_host; time the kernel with events on `stream` and
+ * divide.  ws: 256-B aligned device memory of at least 4 bytes whose first word receives the device
+ * status (see mote_device_status).  n_batches: 1 .. 100000 (about 6 us each). */
+mote_status_t mote_int8_mma_peak(void* ws, int n_batches, double* ops_host, void* stream);
+
 /* Number of kernels the last mote_moe_forward call on this thread enqueued. */
 int mote_last_launch_count(void);
 

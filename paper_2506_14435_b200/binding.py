@@ -83,6 +83,8 @@ lib.mote_device_status.restype = C.c_int
 lib.mote_device_status.argtypes = [C.c_void_p, C.c_void_p]
 lib.mote_selftest_bounded_wait.restype = C.c_int
 lib.mote_selftest_bounded_wait.argtypes = [C.c_void_p, C.c_uint64, C.c_void_p]
+lib.mote_int8_mma_peak.restype = C.c_int
+lib.mote_int8_mma_peak.argtypes = [C.c_void_p, C.c_int, C.POINTER(C.c_double), C.c_void_p]
 lib.mote_last_launch_count.restype = C.c_int
 lib.mote_last_launch_count.argtypes = []
 
@@ -382,3 +384,25 @@ def mote_moe_forward_profile(layer: MoteLayer, x: torch.Tensor, out=None, residu
     _check(lib.mote_moe_forward_profile(C.byref(s), _ptr(x), _ptr(residual), T, _ptr(out), _ptr(ws), ws.numel(),
                                         _stream(), ms), "mote_moe_forward_profile")
     return dict(zip(STAGE_NAMES, [float(v) for v in ms]))
+
+
+def mote_int8_mma_peak(n_batches: int, repeats: int = 5) -> dict:
+    """Times the library's MMA-only kernel (mote_int8_mma_peak) with CUDA events on the current
+    stream, `repeats` launches back to back after one warm-up: returns {"tops_best", "tops_median",
+    "ms" (sorted), "ms_in_order", "ops" (per launch)}."""
+    ws = torch.zeros(256, dtype=torch.uint8, device="cuda")
+    ops = C.c_double(0.0)
+    stream = torch.cuda.current_stream()
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(repeats + 2)]
+    evs[0].record(stream)
+    for i in range(repeats + 1):
+        _check(lib.mote_int8_mma_peak(_ptr(ws), n_batches, C.byref(ops), _stream()), "mote_int8_mma_peak")
+        evs[i + 1].record(stream)
+    torch.cuda.synchronize()
+    times = [evs[i].elapsed_time(evs[i + 1]) for i in range(1, repeats + 1)]
+    _check(lib.mote_device_status(_ptr(ws), _stream()), "mote_int8_mma_peak (device)")
+    in_order = list(times)
+    times.sort()
+    return {"tops_best": ops.value / (times[0] * 1e-3) / 1e12,
+            "tops_median": ops.value / (times[len(times) // 2] * 1e-3) / 1e12, "ms": times,
+            "ms_in_order": in_order, "ops": ops.value}

@@ -25,12 +25,30 @@ def assert_valid_near_tie_pick(pick, logits, k: int):
     assert np.all(sel[:-1] >= sel[1:] - NEAR_TIE_GAP - 1e-12), (pick, sel.tolist())
 
 
-def assert_elementwise_close(got: np.ndarray, ref: np.ndarray, what: str):
-    """Per-element bound beside the Frobenius norm (which one wrong element cannot fail): two bf16
-    roundings (of the shared expert's h, and of the output itself) leave every element within
-    2^-7 of its own magnitude plus 2^-7 of the row's rms."""
-    rms = np.sqrt(np.mean(ref * ref, axis=1, keepdims=True))
-    bound = 2.0 ** -7 * np.abs(ref) + 2.0 ** -7 * rms + 1e-30
+def shared_rounding_sigma(layer_or: dict, x_bits: np.ndarray) -> np.ndarray:
+    """Standard deviation, per output element, of what the one unavoidable intermediate rounding does
+    to the shared expert's output: the kernels hold h = up * SiLU(gate) as bf16, i.e. every h_i is
+    off by a relative error of at most 2^-9 (spread like a uniform variable: deviation 2^-9/sqrt 3),
+    independent between i, so  s_c = sum_i Wd[c,i] h_i  is off by a variable of deviation
+        sigma_c = 2^-9 / sqrt(3) * sqrt( sum_i (Wd[c,i] h_i)^2 ).
+    Evaluated in fp64 from the same inputs the oracle gets (this is test arithmetic, not the oracle)."""
+    x = O.bf16_to_f32(x_bits).astype(np.float64)
+    if layer_or.get("sh_rtn"):
+        Wg, Wu, Wd = (O.rtn_dequant(*layer_or["sh_rtn"][n]) for n in ("gate", "up", "down"))
+    else:
+        Wg, Wu, Wd = (O.bf16_to_f32(layer_or["sh_" + n]).astype(np.float64) for n in ("gate", "up", "down"))
+    g = x @ Wg.T
+    h = (x @ Wu.T) * (g / (1.0 + np.exp(-g)))
+    return 2.0 ** -9 / np.sqrt(3.0) * np.sqrt((h * h) @ (Wd * Wd).T)
+
+
+def assert_elementwise_close(got: np.ndarray, ref: np.ndarray, sigma: np.ndarray, what: str):
+    """Per-element bound beside the Frobenius norm (which one wrong element cannot fail).  The GPU
+    result differs from the fp64 oracle by the rounding of the shared expert's h to bf16 (deviation
+    sigma per element, see shared_rounding_sigma; never more than 8 sigma in practice: the error is a
+    sum of bounded independent terms) and by the final rounding of the value itself (2^-9 relative for
+    a bf16 output; taken as 2^-8 to leave room for the fp32 accumulation order)."""
+    bound = 8.0 * sigma + 2.0 ** -8 * np.abs(ref) + 1e-30
     bad = np.abs(got - ref) > bound
     assert not bad.any(), (what, int(bad.sum()), float(np.max(np.abs(got - ref) / bound)))
 
@@ -102,11 +120,12 @@ def check_forward(mote, layer_gpu, layer_or: dict, x_bits: np.ndarray, residual_
     sh = taps["shared_out"][toks_dev].cpu().numpy().astype(np.float64)
     sh_err = np.linalg.norm(sh - ref["shared_out"]) / max(np.linalg.norm(ref["shared_out"]), 1e-30)
     assert sh_err <= REL_FRO_TOL, sh_err
-    assert_elementwise_close(sh, ref["shared_out"], "shared_out")
+    sigma = shared_rounding_sigma(layer_or, x_bits[toks])
+    assert_elementwise_close(sh, ref["shared_out"], sigma, "shared_out")
     out_f = O.bf16_to_f32(bf16_bits(out[toks_dev])).astype(np.float64)
     err = np.linalg.norm(out_f - ref["out"]) / max(np.linalg.norm(ref["out"]), 1e-30)
     assert err <= REL_FRO_TOL, err
-    assert_elementwise_close(out_f, ref["out"], "out")
+    assert_elementwise_close(out_f, ref["out"], sigma, "out")
     # the launch configuration that is timed passes no taps (other epilogue branches, no fp32 copy
     # of the shared output): it must give the very same bits
     if not out_alias_residual:

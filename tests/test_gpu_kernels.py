@@ -247,3 +247,13 @@ def test_status_word_survives_the_layers_of_a_stack_and_is_cleared_by_the_next_c
     assert mote.lib.mote_device_status(ws.data_ptr(), None) == 0    # cleared at the start of the stack
     assert mote.lib.mote_selftest_bounded_wait(ws.data_ptr(), 1_000_000, None) == 0
     assert mote.lib.mote_device_status(ws.data_ptr(), None) == 7
+
+
+def test_int8_mma_peak_kernel_runs_and_its_time_follows_the_work(mote):
+    from paper_2506_14435_b200.binding import mote_int8_mma_peak
+    a = mote_int8_mma_peak(400)
+    b = mote_int8_mma_peak(800)
+    # twice the MMAs take about twice as long (the kernel really issues them), and the rate is that
+    # of a tensor pipe (far above what CUDA cores can do: 148 SMs x 128 lanes x 2 GHz x 8 = 0.3 POP/s)
+    assert 1.7 < b["ms"][0] / a["ms"][0] < 2.3
+    assert 1000.0 < b["tops_best"] < 6000.0
