@@ -224,7 +224,6 @@ __device__ __forceinline__ float glu_h(int acc_g, int acc_u, float c_g, float c_
   float u = __fmul_rn(i2f_small(acc_u), c_u);
   return __fmul_rn(u, silu_pinned(g));
 }
-
 // The same h through the special-function unit, with a flag telling when that is not enough.
 //   E' = ex2.approx(t), t = fl(-g*log2e) as above (relative error <= 2^-22; the polynomial's E is
 //        within 4e-7 of 2^t)                                     -> |E' - E| <= 6.4e-7 * E

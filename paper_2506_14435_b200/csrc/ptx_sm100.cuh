@@ -79,6 +79,14 @@ __device__ __forceinline__ void tma_load_2d(uint32_t smem_dst, const void* tmap,
       : "memory");
 }
 
+// One 32-byte store per thread (a whole L2 sector; 32-byte aligned address).
+__device__ __forceinline__ void st_global_v8(void* p, uint32_t v0, uint32_t v1, uint32_t v2, uint32_t v3, uint32_t v4,
+                                             uint32_t v5, uint32_t v6, uint32_t v7) {
+  asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p), "r"(v0), "r"(v1), "r"(v2), "r"(v3),
+               "r"(v4), "r"(v5), "r"(v6), "r"(v7)
+               : "memory");
+}
+
 // 2-D tiled store shared -> global (bulk async-group completion).  x must be a multiple of 16
 // bytes worth of elements; neither coordinate may be negative.
 __device__ __forceinline__ void tma_store_2d(const void* tmap, uint32_t smem_src, int x, int y) {

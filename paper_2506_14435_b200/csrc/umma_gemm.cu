@@ -145,6 +145,14 @@ __device__ __forceinline__ void report_abort(volatile int* abort_flag, uint32_t*
   if (*abort_flag) atomicExch(status, 1u);
 }
 
+// glu_h as ONE copy of code.  The gate/up epilogue recomputes about one element in a thousand with
+// the pinned sequence, from a loop unrolled over sixteen elements: sixteen inlined copies of the
+// division and the polynomial cost it instruction cache and scheduling freedom for nothing
+// (8 % of the kernel at K = 896).
+static __device__ __noinline__ float glu_h_rare(int acc_g, int acc_u, float c_g, float c_u) {
+  return glu_h(acc_g, acc_u, c_g, c_u);
+}
+
 // ------------------------------------------------------------------------------------------------
 template <int MODE>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -429,7 +437,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
                 if (redo_mask) {
 #pragma unroll
                   for (int j = 0; j < 16; ++j)
-                    if ((redo_mask >> j) & 1u) hv[j] = glu_h((int)rg[j] - rs, (int)ru[j] - rs, c0, c1);
+                    if ((redo_mask >> j) & 1u) hv[j] = glu_h_rare((int)rg[j] - rs, (int)ru[j] - rs, c0, c1);
                 }
 #pragma unroll
                 for (int j = 0; j < 16; ++j) hmax = fmaxf(hmax, fabsf(hv[j]));
@@ -459,9 +467,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
 #pragma unroll
               for (int j = 0; j < 8; ++j) packed[j] = pack_bf16x2(hv[2 * j], hv[2 * j + 1]);
               if (TR::kTernary) {
-                uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<uint16_t*>(a.out) + row * a.n_out + col0 + c);
-                dst[0] = make_uint4(packed[0], packed[1], packed[2], packed[3]);
-                dst[1] = make_uint4(packed[4], packed[5], packed[6], packed[7]);
+                // the thread's 16 bf16 values are one 32-byte sector of its row: one store
+                st_global_v8(reinterpret_cast<uint16_t*>(a.out) + row * a.n_out + col0 + c, packed[0], packed[1], packed[2],
+                             packed[3], packed[4], packed[5], packed[6], packed[7]);
               } else {
                 uint4* sdst = reinterpret_cast<uint4*>(stg + lane * kPitch + (c - cr) * 2);
                 sdst[0] = make_uint4(packed[0], packed[1], packed[2], packed[3]);
@@ -531,10 +539,12 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
               }
             }
             if (a.out) {
-              float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(a.out) + split * a.split_stride +
-                                                      row * a.n_out + col0 + c);
+              float* dst = reinterpret_cast<float*>(a.out) + split * a.split_stride + row * a.n_out + col0 + c;
 #pragma unroll
-              for (int v = 0; v < 4; ++v) dst[v] = make_float4(o[4 * v], o[4 * v + 1], o[4 * v + 2], o[4 * v + 3]);
+              for (int v = 0; v < 2; ++v)
+                st_global_v8(dst + 8 * v, __float_as_uint(o[8 * v]), __float_as_uint(o[8 * v + 1]), __float_as_uint(o[8 * v + 2]),
+                             __float_as_uint(o[8 * v + 3]), __float_as_uint(o[8 * v + 4]), __float_as_uint(o[8 * v + 5]),
+                             __float_as_uint(o[8 * v + 6]), __float_as_uint(o[8 * v + 7]));
             }
             if (TR::kTernary && a.tap0) {
               int4* t0 = reinterpret_cast<int4*>(a.tap0 + row * a.n_out + col0 + c);
