@@ -87,6 +87,14 @@ __device__ __forceinline__ void st_global_v8(void* p, uint32_t v0, uint32_t v1, 
                : "memory");
 }
 
+// One 32-byte load per thread (32-byte aligned address).
+__device__ __forceinline__ void ld_global_v8(const void* p, uint32_t (&v)[8]) {
+  asm volatile("ld.global.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+               : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+               : "l"(p)
+               : "memory");
+}
+
 // 2-D tiled store shared -> global (bulk async-group completion).  x must be a multiple of 16
 // bytes worth of elements; neither coordinate may be negative.
 __device__ __forceinline__ void tma_store_2d(const void* tmap, uint32_t smem_src, int x, int y) {

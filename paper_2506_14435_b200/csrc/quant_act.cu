@@ -13,6 +13,7 @@
 
 #include "mote_common.cuh"
 #include "mote_internal.h"
+#include "ptx_sm100.cuh"
 
 namespace mote {
 
@@ -166,8 +167,8 @@ __global__ void __launch_bounds__(256) quant_rows_known_beta_kernel(const uint4*
       row = (int)(u / units_per_row);
       const float b = fmaxf(beta[row], kEpsScale);
       const QaScale qs = qa_scale(b);
-      const uint4 r0 = h[u * 2], r1 = h[u * 2 + 1];
-      const uint32_t w[8] = {r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w};
+      uint32_t w[8];
+      ptx::ld_global_v8(h + u * 2, w);            // the unit's 16 bf16 values: one 32-byte load
       uint32_t qv[16];
 #pragma unroll
       for (int j = 0; j < 8; ++j) {

@@ -75,6 +75,7 @@ struct UmmaArgs {
   //   comb_out[t, :] = bf16( s[t, :] + sum_j comb_w[t, j] * comb_y[comb_perm[t*k + j], :] [+ comb_res[t, :]] )
   const float* comb_y; const float* comb_w; const int32_t* comb_perm; const uint16_t* comb_res; uint16_t* comb_out;
   int comb_k;
+  int comb_wide;            // comb_res and comb_out are 32-byte aligned (the caller only promises 16): 32-byte accesses
 };
 
 struct __align__(8) PipeBarriers {
@@ -557,30 +558,36 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
 #pragma unroll
               for (int j = 0; j < MOTE_MAX_TOPK; ++j)
                 if (j < a.comb_k) {
-                  const float4* yp = reinterpret_cast<const float4*>(cy[j] + c);
 #pragma unroll
-                  for (int v = 0; v < 4; ++v) {
-                    const float4 yv = yp[v];
-                    o[4 * v] = fmaf(cw[j], yv.x, o[4 * v]);         o[4 * v + 1] = fmaf(cw[j], yv.y, o[4 * v + 1]);
-                    o[4 * v + 2] = fmaf(cw[j], yv.z, o[4 * v + 2]); o[4 * v + 3] = fmaf(cw[j], yv.w, o[4 * v + 3]);
+                  for (int v = 0; v < 2; ++v) {
+                    uint32_t yv[8];
+                    ld_global_v8(cy[j] + c + 8 * v, yv);
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) o[8 * v + u] = fmaf(cw[j], __uint_as_float(yv[u]), o[8 * v + u]);
                   }
                 }
               if (a.comb_res) {
-                const uint4* rp = reinterpret_cast<const uint4*>(a.comb_res + row * a.n_out + col0 + c);
-#pragma unroll
-                for (int v = 0; v < 2; ++v) {
-                  const uint4 r = rp[v];
-                  const uint32_t rw[4] = {r.x, r.y, r.z, r.w};
-#pragma unroll
-                  for (int u = 0; u < 4; ++u) { o[8 * v + 2 * u] += bf16_lo(rw[u]); o[8 * v + 2 * u + 1] += bf16_hi(rw[u]); }
+                uint32_t rw[8];
+                if (a.comb_wide) {
+                  ld_global_v8(a.comb_res + row * a.n_out + col0 + c, rw);
+                } else {
+                  const uint4* rp = reinterpret_cast<const uint4*>(a.comb_res + row * a.n_out + col0 + c);
+                  const uint4 r0 = rp[0], r1 = rp[1];
+                  rw[0] = r0.x; rw[1] = r0.y; rw[2] = r0.z; rw[3] = r0.w; rw[4] = r1.x; rw[5] = r1.y; rw[6] = r1.z; rw[7] = r1.w;
                 }
+#pragma unroll
+                for (int u = 0; u < 8; ++u) { o[2 * u] += bf16_lo(rw[u]); o[2 * u + 1] += bf16_hi(rw[u]); }
               }
               uint32_t pk[8];
 #pragma unroll
               for (int v = 0; v < 8; ++v) pk[v] = f32_to_bf16_bits(o[2 * v]) | (f32_to_bf16_bits(o[2 * v + 1]) << 16);
-              uint4* od = reinterpret_cast<uint4*>(a.comb_out + row * a.n_out + col0 + c);
-              od[0] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-              od[1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+              if (a.comb_wide) {
+                st_global_v8(a.comb_out + row * a.n_out + col0 + c, pk[0], pk[1], pk[2], pk[3], pk[4], pk[5], pk[6], pk[7]);
+              } else {
+                uint4* od = reinterpret_cast<uint4*>(a.comb_out + row * a.n_out + col0 + c);
+                od[0] = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                od[1] = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+              }
             }
           }
         }
@@ -783,6 +790,7 @@ mote_status_t launch_shared_umma(const void* act, const SharedMat& w0, const Sha
     a.comb_y = comb->y; a.comb_w = comb->w; a.comb_perm = comb->perm;
     a.comb_res = static_cast<const uint16_t*>(comb->residual); a.comb_out = static_cast<uint16_t*>(comb->out);
     a.comb_k = comb->k;
+    a.comb_wide = ((reinterpret_cast<uintptr_t>(comb->out) | reinterpret_cast<uintptr_t>(comb->residual)) & 31u) == 0;
   }
   const int max_items = max_mtiles * a.n_ntiles * a.k_splits;
   if (bits == 8)

@@ -231,3 +231,25 @@ def test_rtn_prefill_expanding_once_or_inside_the_gemm_agree(mote, bits):
     out2 = mote.mote_moe_forward(layer_q, x)
     torch.cuda.synchronize()
     assert torch.equal(out1, out2)
+
+
+@pytest.mark.parametrize("T", [5, 200])
+def test_output_and_residual_aligned_to_16_bytes_only(mote, T):
+    # the C ABI promises kernels nothing beyond 16-byte alignment of out and residual: a view that
+    # starts 16 bytes into an allocation must give the bits of the aligned call (the tensor path's
+    # fused combine uses 32-byte accesses only where the pointers allow them)
+    wl = synth.custom("align", 128, 256, 4, 2, T, 4400, w_std=0.08)
+    layer = mote.MoteLayer.from_master(synth.master_layer(wl))
+    x = bf16_tensor(synth.tokens(wl))
+    res = bf16_tensor(synth.tokens(wl, stream=1))
+    want = mote.mote_moe_forward(layer, x, residual=res)
+    n = T * wl.d
+    res_buf = torch.empty(n + 8, dtype=torch.bfloat16, device="cuda")
+    out_buf = torch.empty(n + 8, dtype=torch.bfloat16, device="cuda")
+    res16 = res_buf[8:].view(T, wl.d)
+    out16 = out_buf[8:].view(T, wl.d)
+    res16.copy_(res)
+    assert res16.data_ptr() % 32 == 16 and out16.data_ptr() % 32 == 16
+    got = mote.mote_moe_forward(layer, x, residual=res16, out=out16)
+    torch.cuda.synchronize()
+    assert torch.equal(got, want)
