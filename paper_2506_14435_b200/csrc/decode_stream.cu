@@ -879,11 +879,12 @@ __device__ __forceinline__ void down_tile_done(const DecodeDownArgs& a, int tile
 }
 
 // up to 16 tokens: two CTAs per SM (at most 64 registers; at 78 registers the 16-token kernel had
-// one CTA per SM and was 8-15 % slower; the one-tile kernels of the RTN widths are capped too, the
-// bf16 one needs 64 anyway.  The 16-token 4-bit expansion would spill too much under that cap.)
+// one CTA per SM and was 8-15 % slower; every one-tile kernel is capped too: left alone the bf16 one
+// takes 106 registers, one CTA per SM, and the step is 5-10 % slower.  The 16-token 4-bit expansion
+// would spill too much under that cap.)
 template <int NTB, int kShBits>
 __global__ void __launch_bounds__(kDownWarps * 32,
-                                  ((NTB == 1 && kShBits != 16) || (NTB == 2 && kShBits != 4)) ? 2 : 1)
+                                  (NTB == 1 || (NTB == 2 && kShBits != 4)) ? 2 : 1)
 decode_down_kernel(DecodeDownArgs a) {
   __shared__ ExpertList s_list;
   __shared__ int s_last;
