@@ -58,6 +58,12 @@ def test_c1_full_parity(mote, path):
     (256, 512, 4, 2, 64, dict(bias="zipf"), STREAM),      # the largest batch, uneven expert loads
     (192, 320, 8, 1, 33, dict(norm_topk=0), STREAM),
     (128, 256, 64, 8, 37, {}, STREAM),                    # many experts, k = 8
+    # a handful of pairs
+    (256, 512, 4, 2, 2, {}, STREAM),                      # two tokens, top-2
+    (128, 256, 2, 1, 3, dict(norm_topk=0), STREAM),       # three pairs on two experts
+    (128, 320, 8, 4, 1, {}, STREAM),                      # one token, k = 4
+    (896, 4864, 4, 2, 2, dict(outlier_frac=0.01), STREAM),
+    (192, 320, 1, 1, 4, {}, STREAM),                      # one expert takes all four rows
 ])
 def test_small_shapes(mote, d, f, E, k, T, kw, path):
     wl = synth.custom("small", d, f, E, k, T, 2000 + d + f + T, **kw)
