@@ -2,9 +2,9 @@
 //
 // Three launches per matrix:
 //   1. abs_sum_bins    exact accumulation of sum |w|: each fp32 magnitude is split into its
-//                      24-bit integer significand and its exponent; significands are added into
-//                      one 64-bit integer bin per exponent.  Integer adds commute, so the bins do
-//                      not depend on thread order.
+//                      24-bit integer significand and its exponent; significands are added (shifted
+//                      to a common unit, as integers) into 64-bit integer bins indexed by exponent.
+//                      Integer adds commute, so the bins' total does not depend on thread order.
 //   2. alpha_finalize  one thread adds the bins into a 384-bit integer (exact), rounds it to
 //                      fp64 (nearest even), divides by m*n in fp64 and rounds once to fp32.
 //   3. pack_codes      code = clamp(rint(w / alpha), -1, 1), four codes per byte.
@@ -17,6 +17,48 @@ namespace mote {
 
 constexpr int kBins = 256;
 
+// Exact sum of |w| without a warp vote per element: every thread keeps ONE 64-bit fixed-point
+// accumulator in units of 2^(base - 150), where `base` is an exponent it picks from its first
+// non-zero element (16 binades below it).  An element with exponent e in [base, base + 31] adds
+// significand << (e - base), below 2^55, so some five hundred elements fit before a flush is needed;
+// the grid gives a thread far fewer, and the flush is made anyway every 256 additions (and when a larger element moves the window up).  A flush adds
+// the low 32 bits to bin `base` and the high 32 bits to bin `base + 32` (whose unit is 2^32 times
+// larger): exact, and every bin stays far below 2^64.  The rare element outside the window goes
+// straight to the bin of its own exponent.  All of it is integer addition, so neither the choice of
+// base nor the order of threads changes the bins' total.
+struct AbsAcc {
+  unsigned long long acc;
+  int base, count;
+};
+
+__device__ __forceinline__ void abs_acc_flush(AbsAcc& st, unsigned long long* sbins) {
+  if (st.acc) {
+    atomicAdd(&sbins[st.base], st.acc & 0xFFFFFFFFull);
+    if (st.acc >> 32) atomicAdd(&sbins[st.base + 32], st.acc >> 32);
+  }
+  st.acc = 0ull;
+  st.count = 0;
+}
+
+__device__ __forceinline__ void abs_acc_add(AbsAcc& st, uint32_t bits, unsigned long long* sbins) {
+  const uint32_t a = bits & 0x7FFFFFFFu;
+  if (a == 0u) return;
+  const uint32_t e_raw = a >> 23;
+  const uint32_t mant = e_raw ? ((a & 0x7FFFFFu) | 0x800000u) : a;   // subnormals: no hidden bit
+  const int e = e_raw ? (int)e_raw : 1;                              // ... and the unit of exponent 1
+  if (st.base < 0 || e > st.base + 31) {                             // first element, or one above the window:
+    if (st.base >= 0) abs_acc_flush(st, sbins);                      // move the window up to it
+    st.base = min(max(e - 16, 1), 222);                              // base + 32 must be a valid bin
+  }
+  const unsigned sh = (unsigned)(e - st.base);
+  if (sh < 32u) {
+    st.acc += (unsigned long long)mant << sh;
+    if (++st.count == 256) abs_acc_flush(st, sbins);
+  } else {
+    atomicAdd(&sbins[e_raw], (unsigned long long)mant);              // outside the window: its own bin
+  }
+}
+
 template <bool kBf16>
 __global__ void __launch_bounds__(256) abs_sum_bins_kernel(const void* __restrict__ W, int64_t n_vec,
                                                            unsigned long long* __restrict__ bins) {
@@ -24,35 +66,29 @@ __global__ void __launch_bounds__(256) abs_sum_bins_kernel(const void* __restric
   for (int i = threadIdx.x; i < kBins; i += blockDim.x) sbins[i] = 0ull;
   __syncthreads();
 
-  const int lane = threadIdx.x & 31;
-  // one "vec" = 4 elements (a float4, or 4 bf16 = uint2)
+  // one "vec" = 4 elements (a float4, or 4 bf16 = uint2); two vecs in flight per thread
   const int64_t stride = int64_t(gridDim.x) * blockDim.x;
-  const int64_t first = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
-  // all lanes of a warp run the same number of iterations so the warp-wide votes stay converged
-  const int64_t warp_first = first - lane;
-  for (int64_t base = warp_first; base < n_vec; base += stride) {
-    const int64_t v = base + lane;
-    uint32_t bits[4] = {0u, 0u, 0u, 0u};
-    if (v < n_vec) {
-      if (kBf16) {
-        uint2 r = reinterpret_cast<const uint2*>(W)[v];
-        bits[0] = r.x << 16; bits[1] = r.x & 0xFFFF0000u; bits[2] = r.y << 16; bits[3] = r.y & 0xFFFF0000u;
-      } else {
-        uint4 r = reinterpret_cast<const uint4*>(W)[v];
-        bits[0] = r.x; bits[1] = r.y; bits[2] = r.z; bits[3] = r.w;
+  AbsAcc st{0ull, -1, 0};
+  for (int64_t v = int64_t(blockIdx.x) * blockDim.x + threadIdx.x; v < n_vec; v += 2 * stride) {
+    uint32_t bits[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      const int64_t vv = v + u * stride;
+      if (vv < n_vec) {
+        if (kBf16) {
+          const uint2 r = reinterpret_cast<const uint2*>(W)[vv];
+          bits[4 * u] = r.x << 16; bits[4 * u + 1] = r.x & 0xFFFF0000u;
+          bits[4 * u + 2] = r.y << 16; bits[4 * u + 3] = r.y & 0xFFFF0000u;
+        } else {
+          const uint4 r = reinterpret_cast<const uint4*>(W)[vv];
+          bits[4 * u] = r.x; bits[4 * u + 1] = r.y; bits[4 * u + 2] = r.z; bits[4 * u + 3] = r.w;
+        }
       }
     }
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const uint32_t a = bits[j] & 0x7FFFFFFFu;
-      const uint32_t e = a >> 23;
-      const uint32_t mant = e ? ((a & 0x7FFFFFu) | 0x800000u) : a;   // subnormals: no hidden bit
-      // lanes with the same exponent add their significands first (sum < 2^29)
-      const uint32_t peers = __match_any_sync(0xffffffffu, e);
-      const uint32_t sum = __reduce_add_sync(peers, mant);
-      if (lane == (__ffs(peers) - 1) && sum) atomicAdd(&sbins[e], (unsigned long long)sum);
-    }
+    for (int j = 0; j < 8; ++j) abs_acc_add(st, bits[j], sbins);
   }
+  abs_acc_flush(st, sbins);
   __syncthreads();
   for (int i = threadIdx.x; i < kBins; i += blockDim.x)
     if (sbins[i]) atomicAdd(&bins[i], sbins[i]);
@@ -62,12 +98,17 @@ __global__ void __launch_bounds__(256) abs_sum_bins_kernel(const void* __restric
 // of 2^-149.
 __global__ void alpha_finalize_kernel(const unsigned long long* __restrict__ bins, double count,
                                       float* __restrict__ alpha) {
+  // the warp fetches the bins together (one round trip instead of 255 dependent ones) ...
+  __shared__ unsigned long long s_bins[kBins];
+  for (int i = threadIdx.x; i < kBins; i += blockDim.x) s_bins[i] = bins[i];
+  __syncthreads();
   if (threadIdx.x != 0 || blockIdx.x != 0) return;
+  // ... and one thread adds them up
   constexpr int kLimbs = 12;
   uint32_t L[kLimbs];
   for (int i = 0; i < kLimbs; ++i) L[i] = 0u;
   for (int e = 0; e < 255; ++e) {            // e = 255 (inf/nan) is undefined input, ignored
-    const unsigned long long v = bins[e];
+    const unsigned long long v = s_bins[e];
     if (!v) continue;
     const int s = (e ? e : 1) - 1;
     const int wo = s >> 5, bo = s & 31;
