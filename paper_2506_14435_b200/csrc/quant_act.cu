@@ -221,48 +221,117 @@ __global__ void __launch_bounds__(256, 4) quant_act_rows_kernel(QuantActArgs a) 
 }
 
 // Q_a(h) when the row maxima are already known (the gate/up GEMM epilogue accumulates them with
-// atomicMax): a pure streaming pass, one unit of 16 elements per thread and iteration.
-__global__ void __launch_bounds__(256) quant_rows_known_beta_kernel(const uint4* __restrict__ h, int64_t n_units_total,
-                                                                    int units_per_row, uint4* __restrict__ q,
-                                                                    float* beta, int32_t* __restrict__ rowsum,
-                                                                    int interleave, int early_trigger) {
+// atomicMax): a pure streaming pass.  A work item is a run of `seg_units` 16-element units of one
+// row; a warp takes items round-robin and its lanes take the run's units 32 bytes at a time, two
+// loads in flight per lane.  Row, scale and the row sum are handled once per item, not per unit.
+//
+// Eq. 8 for one unit of 16 elements: the division-free form (r = x * c, c = fl(127 * fl(1/beta)))
+// per element, which needs the division only where r is within 2^-14 of a
+// half-integer: |r - 127x/beta| <= 127 * 3 * 2^-24 and |fl(fl(127x)/beta) - 127x/beta| <= 127 * 2^-24
+// add up to 3.03e-5 < 2^-14, so outside that band both round to the same integer.  A unit with such
+// an element (one in 500) is redone by an out-of-line function, so that the streaming loop holds
+// neither the division's instructions nor a branch per element: 9.4 instead of 20 instructions per
+// element.  (The two kernels above keep the branch per element: with the out-of-line call the
+// row-staging kernel spills and drops from 3.5 to 2.9 TB/s, and the scatter kernel gains at
+// T = 8192 what it loses at T <= 4096, under 0.4 % of the layer either way.)
+constexpr float kQaFastBand = 0.49993896484375f;   // 0.5 - 2^-14
+
+__device__ __forceinline__ uint4 pack_unit(const uint32_t (&qv)[16], int interleave) {
+  uint32_t o[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+    o[i] = interleave ? pack_low_bytes(qv[i], qv[4 + i], qv[8 + i], qv[12 + i])
+                      : pack_low_bytes(qv[4 * i], qv[4 * i + 1], qv[4 * i + 2], qv[4 * i + 3]);
+  return make_uint4(o[0], o[1], o[2], o[3]);
+}
+
+// `band` is kQaFastBand, or a negative number for a row whose scale is outside the range in which
+// the division-free form is valid (every element then takes the division).
+__device__ __forceinline__ float qa_band(const QaScale& s) { return s.fast ? kQaFastBand : -1.0f; }
+
+__device__ __noinline__ uint4 quant_unit_exact(uint4 wa, uint4 wb, float beta, float c, float band, int interleave) {
+  const uint32_t w[8] = {wa.x, wa.y, wa.z, wa.w, wb.x, wb.y, wb.z, wb.w};
+  uint32_t qv[16];
+#pragma unroll
+  for (int j = 0; j < 16; ++j) {
+    const float x = (j & 1) ? bf16_hi(w[j >> 1]) : bf16_lo(w[j >> 1]);
+    const float r = __fmul_rn(x, c);
+    const float m = __fadd_rn(r, kMagic);
+    const float frac = __fsub_rn(r, __fsub_rn(m, kMagic));
+    qv[j] = (fabsf(frac) < band) ? __float_as_uint(m) : (uint32_t)quant_one(x, beta);
+  }
+  return pack_unit(qv, interleave);
+}
+
+// The unit's 16 codes, packed (plain or interleaved byte order).
+__device__ __forceinline__ uint4 quant_unit(uint4 wa, uint4 wb, float beta, float c, float band, int interleave) {
+  const uint32_t w[8] = {wa.x, wa.y, wa.z, wa.w, wb.x, wb.y, wb.z, wb.w};
+  uint32_t qv[16];
+  bool exact = false;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const float r0 = __fmul_rn(bf16_lo(w[j]), c), r1 = __fmul_rn(bf16_hi(w[j]), c);
+    const float m0 = __fadd_rn(r0, kMagic), m1 = __fadd_rn(r1, kMagic);
+    const float f0 = __fsub_rn(r0, __fsub_rn(m0, kMagic)), f1 = __fsub_rn(r1, __fsub_rn(m1, kMagic));
+    qv[2 * j] = __float_as_uint(m0);
+    qv[2 * j + 1] = __float_as_uint(m1);
+    exact = exact || !(fabsf(f0) < band) || !(fabsf(f1) < band);
+  }
+  uint4 o = pack_unit(qv, interleave);
+  if (exact) o = quant_unit_exact(wa, wb, beta, c, band, interleave);
+  return o;
+}
+
+// sum of the 16 codes of a packed unit
+__device__ __forceinline__ int unit_sum(uint4 o) {
+  int sum = __dp4a((int)o.x, 0x01010101, 0);
+  sum = __dp4a((int)o.y, 0x01010101, sum);
+  sum = __dp4a((int)o.z, 0x01010101, sum);
+  return __dp4a((int)o.w, 0x01010101, sum);
+}
+
+__global__ void __launch_bounds__(256) quant_rows_known_beta_kernel(const uint4* __restrict__ h, int64_t n_items,
+                                                                    int units_per_row, int seg_units, int nseg,
+                                                                    uint4* __restrict__ q, float* beta,
+                                                                    int32_t* __restrict__ rowsum, int interleave,
+                                                                    int early_trigger) {
   const int lane = threadIdx.x & 31;
-  const int64_t stride = int64_t(gridDim.x) * blockDim.x;
-  const int64_t first = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
+  const int64_t n_warps = (int64_t(gridDim.x) * blockDim.x) >> 5;
   pdl_wait();                            // no-op unless launched as a programmatic dependent
   // decode path: the down kernel may start on work that does not need this kernel's output.  (Not
   // for the tensor path: its persistent GEMM CTAs would take this kernel's registers away.)
   if (early_trigger) pdl_trigger();
-  for (int64_t base = first - lane; base < n_units_total; base += stride) {
-    const int64_t u = base + lane;
-    const bool ok = u < n_units_total;
-    int row = -1, sum = 0;
-    if (ok) {
-      row = (int)(u / units_per_row);
-      const float b = fmaxf(beta[row], kEpsScale);
-      const QaScale qs = qa_scale(b);
-      uint32_t w[8];
-      ptx::ld_global_v8(h + u * 2, w);            // the unit's 16 bf16 values: one 32-byte load
-      uint32_t qv[16];
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        qv[2 * j] = quant_byte(bf16_lo(w[j]), qs);
-        qv[2 * j + 1] = quant_byte(bf16_hi(w[j]), qs);
+  for (int64_t item = (int64_t(blockIdx.x) * blockDim.x + threadIdx.x) >> 5; item < n_items; item += n_warps) {
+    const int row = (int)(item / nseg);
+    const int seg = (int)(item - int64_t(row) * nseg);
+    const int u_end = min((seg + 1) * seg_units, units_per_row);
+    const float b = fmaxf(beta[row], kEpsScale);
+    const QaScale qs = qa_scale(b);
+    const float band = qa_band(qs);
+    const uint4* hr = h + int64_t(row) * units_per_row * 2;
+    uint4* qr = q + int64_t(row) * units_per_row;
+    int sum = 0;
+    for (int u = seg * seg_units + lane; u < u_end; u += 64) {
+      const bool second = u + 32 < u_end;
+      uint32_t w0[8], w1[8];
+      ptx::ld_global_v8(hr + u * 2, w0);            // a unit's 16 bf16 values: one 32-byte load
+      if (second) ptx::ld_global_v8(hr + (u + 32) * 2, w1);
+      const uint4 o0 = quant_unit(make_uint4(w0[0], w0[1], w0[2], w0[3]), make_uint4(w0[4], w0[5], w0[6], w0[7]), b,
+                                  qs.c, band, interleave);
+      qr[u] = o0;
+      sum += unit_sum(o0);
+      if (second) {
+        const uint4 o1 = quant_unit(make_uint4(w1[0], w1[1], w1[2], w1[3]), make_uint4(w1[4], w1[5], w1[6], w1[7]), b,
+                                    qs.c, band, interleave);
+        qr[u + 32] = o1;
+        sum += unit_sum(o1);
       }
-      uint32_t o[4];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        o[i] = interleave ? pack_low_bytes(qv[i], qv[4 + i], qv[8 + i], qv[12 + i])
-                          : pack_low_bytes(qv[4 * i], qv[4 * i + 1], qv[4 * i + 2], qv[4 * i + 3]);
-        sum = __dp4a((int)o[i], 0x01010101, sum);
-      }
-      q[u] = make_uint4(o[0], o[1], o[2], o[3]);
-      if (u - int64_t(row) * units_per_row == 0) beta[row] = b;   // publish the clamped scale
     }
-    // one atomic per (warp, row)
-    const unsigned peers = __match_any_sync(0xffffffffu, row);
-    const int total = __reduce_add_sync(peers, sum);
-    if (ok && lane == (__ffs(peers) - 1)) atomicAdd(rowsum + row, total);
+    sum = __reduce_add_sync(0xffffffffu, sum);
+    if (lane == 0) {
+      atomicAdd(rowsum + row, sum);
+      if (seg == 0) beta[row] = b;                  // publish the clamped scale
+    }
   }
 }
 
@@ -271,15 +340,26 @@ mote_status_t launch_quant_rows_known_beta(const void* h_bf16, int64_t rows, int
                                            bool early_trigger) {
   if (rows == 0) return MOTE_OK;
   const int units_per_row = n / 16;
-  const int64_t total = rows * units_per_row;
-  const unsigned blocks = (unsigned)std::min<int64_t>((total + 255) / 256, 148 * 8);
+  // Runs of equal length, 32 units at least, and about four times as many warps as are resident at
+  // once, two runs each: measured against one resident wave of longer-lived warps (8 % slower at
+  // T = 8192, f = 11008) and against shorter runs (one load round per run: 5-25 % slower).
+  const int64_t target_warps = int64_t(device_sm_count()) * 256;
+  const int max_seg = (units_per_row + 31) / 32;
+  int nseg = (int)std::min<int64_t>(std::max<int64_t>((target_warps + rows - 1) / rows, 1), max_seg);
+  const int seg_units = (units_per_row + nseg - 1) / nseg;
+  nseg = (units_per_row + seg_units - 1) / seg_units;
+  const int64_t items = rows * nseg;
+  const int64_t per_warp = (items + target_warps - 1) / target_warps;
+  const int64_t warps = (items + per_warp - 1) / per_warp;
+  const unsigned blocks = (unsigned)((warps + 7) / 8);
   if (pdl)
     MOTE_CUDA_OK(launch_pdl(quant_rows_known_beta_kernel, dim3(blocks), dim3(256), 0, stream,
-                            static_cast<const uint4*>(h_bf16), total, units_per_row, reinterpret_cast<uint4*>(q), beta,
-                            rowsum, interleave, early_trigger ? 1 : 0));
+                            static_cast<const uint4*>(h_bf16), items, units_per_row, seg_units, nseg,
+                            reinterpret_cast<uint4*>(q), beta, rowsum, interleave, early_trigger ? 1 : 0));
   else
-    quant_rows_known_beta_kernel<<<blocks, 256, 0, stream>>>(static_cast<const uint4*>(h_bf16), total, units_per_row,
-                                                             reinterpret_cast<uint4*>(q), beta, rowsum, interleave, 0);
+    quant_rows_known_beta_kernel<<<blocks, 256, 0, stream>>>(static_cast<const uint4*>(h_bf16), items, units_per_row,
+                                                             seg_units, nseg, reinterpret_cast<uint4*>(q), beta,
+                                                             rowsum, interleave, 0);
   ++g_launch_count;
   MOTE_LAUNCH_OK();
   return MOTE_OK;
