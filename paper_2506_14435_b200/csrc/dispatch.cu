@@ -114,14 +114,34 @@ __global__ void __launch_bounds__(kDispatchThreads) dispatch_kernel(const int32_
 
 // ------------------------------------------------------------------------------------------------
 // Block-wise dispatch for long prefills.  The router leaves, for every block of kRouteBlockTokens
-// tokens, the number of its pairs per expert (blk_hist[n_blk][E]).  This kernel turns them into
-//   offsets[E+1]          first sorted row of every expert
-//   blk_base[n_blk][E]    first sorted row of the block's pairs of that expert
+// tokens, the number of its pairs per expert (blk_hist[E][blk_stride(n_blk)]).  This kernel turns
+// them into
+//   offsets[E+1]                      first sorted row of every expert
+//   blk_base[E][blk_stride(n_blk)]    first sorted row of the block's pairs of that expert
 // (experts outermost, blocks in order: the same stable order as above) and writes the tile tables.
 // The rank of a pair inside its block is recomputed by the activation quantizer, which then knows
 // the sorted row of every pair without a pass of its own.  One CTA, one warp per expert: lane l
-// sums a contiguous range of blocks, a shuffle scan orders the ranges, a second walk writes the bases.
+// sums 16 consecutive blocks (four 16-byte loads), a shuffle scan orders the lanes, a second walk
+// writes the bases.  (With the counts block-major, every load and store of a warp touched 32
+// separate sectors: 18 us at 512 blocks x 16 experts, 11 of them in the second walk.)
 // ------------------------------------------------------------------------------------------------
+constexpr int kScanPer = 16;                           // blocks per lane and chunk
+
+// the lane's 16 counts of chunk c0, zero beyond n_blk
+__device__ __forceinline__ void load_counts(const int32_t* __restrict__ row, int c0, int lane, int n_blk, int (&v)[kScanPer]) {
+  const int b0 = c0 + lane * kScanPer;
+#pragma unroll
+  for (int i = 0; i < kScanPer / 4; ++i) {
+    const int b = b0 + 4 * i;
+    int4 t = make_int4(0, 0, 0, 0);
+    if (b < n_blk) t = *reinterpret_cast<const int4*>(row + b);     // the padded row holds b .. b + 3
+    v[4 * i] = t.x;
+    v[4 * i + 1] = b + 1 < n_blk ? t.y : 0;
+    v[4 * i + 2] = b + 2 < n_blk ? t.z : 0;
+    v[4 * i + 3] = b + 3 < n_blk ? t.w : 0;
+  }
+}
+
 __global__ void __launch_bounds__(kDispatchThreads) dispatch_scan_kernel(const int32_t* __restrict__ blk_hist, int n_blk,
                                                                          int E, int32_t* __restrict__ offsets,
                                                                          int32_t* __restrict__ blk_base,
@@ -130,7 +150,7 @@ __global__ void __launch_bounds__(kDispatchThreads) dispatch_scan_kernel(const i
   __shared__ int s_count[MOTE_MAX_EXPERTS];
   __shared__ int s_first[MOTE_MAX_EXPERTS];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  constexpr int kPer = 16;                             // blocks per lane and chunk: 16 independent loads
+  const int stride = blk_stride(n_blk);
   pdl_wait();                                          // the router's block counts are complete
   // totals per expert (two rounds of 32 warps cover MOTE_MAX_EXPERTS = 64)
 #pragma unroll
@@ -138,15 +158,11 @@ __global__ void __launch_bounds__(kDispatchThreads) dispatch_scan_kernel(const i
     const int e = warp + 32 * r;
     if (e < E) {
       int tot = 0;
-      for (int c0 = 0; c0 < n_blk; c0 += 32 * kPer) {
-        int v[kPer];
+      for (int c0 = 0; c0 < n_blk; c0 += 32 * kScanPer) {
+        int v[kScanPer];
+        load_counts(blk_hist + size_t(e) * stride, c0, lane, n_blk, v);
 #pragma unroll
-        for (int i = 0; i < kPer; ++i) {
-          const int b = c0 + lane * kPer + i;
-          v[i] = b < n_blk ? blk_hist[b * E + e] : 0;
-        }
-#pragma unroll
-        for (int i = 0; i < kPer; ++i) tot += v[i];
+        for (int i = 0; i < kScanPer; ++i) tot += v[i];
       }
       tot = warp_sum(tot);
       if (lane == 0) s_count[e] = tot;
@@ -183,15 +199,13 @@ __global__ void __launch_bounds__(kDispatchThreads) dispatch_scan_kernel(const i
     const int e = warp + 32 * r;
     if (e < E) {
       int carry = s_first[e];
-      for (int c0 = 0; c0 < n_blk; c0 += 32 * kPer) {
-        int v[kPer];
+      int32_t* out = blk_base + size_t(e) * stride;
+      for (int c0 = 0; c0 < n_blk; c0 += 32 * kScanPer) {
+        int v[kScanPer];
+        load_counts(blk_hist + size_t(e) * stride, c0, lane, n_blk, v);
         int tot = 0;
 #pragma unroll
-        for (int i = 0; i < kPer; ++i) {
-          const int b = c0 + lane * kPer + i;
-          v[i] = b < n_blk ? blk_hist[b * E + e] : 0;
-          tot += v[i];
-        }
+        for (int i = 0; i < kScanPer; ++i) tot += v[i];
         int incl = tot;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -199,11 +213,15 @@ __global__ void __launch_bounds__(kDispatchThreads) dispatch_scan_kernel(const i
           if (lane >= o) incl += n;
         }
         int run = carry + incl - tot;
+        const int b0 = c0 + lane * kScanPer;
 #pragma unroll
-        for (int i = 0; i < kPer; ++i) {
-          const int b = c0 + lane * kPer + i;
-          if (b < n_blk) blk_base[b * E + e] = run;
-          run += v[i];
+        for (int i = 0; i < kScanPer / 4; ++i) {
+          int4 t;
+          t.x = run; run += v[4 * i];
+          t.y = run; run += v[4 * i + 1];
+          t.z = run; run += v[4 * i + 2];
+          t.w = run; run += v[4 * i + 3];
+          if (b0 + 4 * i < n_blk) *reinterpret_cast<int4*>(out + b0 + 4 * i) = t;   // the padded row has room
         }
         carry += __shfl_sync(0xffffffffu, incl, 31);
       }

@@ -72,8 +72,8 @@ static Plan make_plan(int d, int f, int E, int k, int64_t T) {
   p.tiles_routed = take((1 + P / 128 + E) * 16);
   p.tiles_shared = take((1 + (size_t(T) + 127) / 128) * 16);
   const size_t n_blk = (size_t(T) + kRouteBlockTokens - 1) / kRouteBlockTokens;
-  p.blk_hist = take(n_blk * E * 4);
-  p.blk_base = take(n_blk * E * 4);
+  p.blk_hist = take(size_t(blk_stride((int)n_blk)) * E * 4);
+  p.blk_base = take(size_t(blk_stride((int)n_blk)) * E * 4);
   p.total = off;
   p.sh_codes_bf16 = take(T >= kExpandMinTokens ? size_t(3) * d * f * 2 : 1);
   p.total_expanded = T >= kExpandMinTokens ? off : p.total;
@@ -361,7 +361,7 @@ extern "C" mote_status_t mote_moe_forward(const mote_layer_t* L, const void* x, 
   qa.x = x; qa.T = T; qa.d = d; qa.ldx = d; qa.q = qx; qa.beta = beta_x; qa.rowsum = rowsum_x;
   qa.perm = perm; qa.k = k; qa.interleave = interleave;
   if (blockwise) {
-    qa.topk_idx = topk_idx; qa.blk_base = blk_base; qa.E = E; qa.perm_out = perm; qa.inv_out = inv;
+    qa.topk_idx = topk_idx; qa.blk_base = blk_base; qa.E = E; qa.n_blk = n_blk; qa.perm_out = perm; qa.inv_out = inv;
     qa.zero_u32 = reinterpret_cast<uint32_t*>(beta_h); qa.zero_i32 = rowsum_h;
   }
   const bool pdl = blockwise;    // from here on every kernel is a programmatic dependent of the one before

@@ -19,7 +19,7 @@ struct QuantActArgs {
   const int32_t* perm;  // scatter variant: pair (t*k+j) -> destination row (when blk_base is null)
   // scatter variant with the block-wise dispatch: the destination row is derived here from the
   // top-k indices and the per-block bases, and written to perm_out / inv_out
-  const int32_t* topk_idx; const int32_t* blk_base; int E;
+  const int32_t* topk_idx; const int32_t* blk_base; int E; int n_blk;
   int32_t* perm_out; int32_t* inv_out;
   uint32_t* zero_u32; int32_t* zero_i32;   // optional [rows] arrays cleared at every destination row
   int k;
@@ -30,8 +30,13 @@ mote_status_t launch_quant_act(const QuantActArgs& a, bool scatter, cudaStream_t
 
 // Router (Eq. 3).  Arguments as mote_route_topk.
 // blk_hist (optional, written only by the tensor-core kernel, i.e. when d % 32 == 0):
-// [ceil(T / kRouteBlockTokens)][E] pairs per expert of every block of tokens.
+// [E][blk_stride(n_blk)] pairs per expert of every block of kRouteBlockTokens tokens, n_blk =
+// ceil(T / kRouteBlockTokens); expert-major, so that the scan reads an expert's counts contiguously.
 constexpr int kRouteBlockTokens = 16;
+#ifdef __CUDACC__
+__host__ __device__
+#endif
+constexpr int blk_stride(int n_blk) { return (n_blk + 3) & ~3; }   // rows start on 16-byte boundaries
 mote_status_t launch_route_topk(const void* x, int64_t T, int d, const float* Wr, const float* bias,
                                 int E, int k, int norm_topk, int32_t* idx, float* w, float* logits,
                                 int32_t* blk_hist, cudaStream_t stream);

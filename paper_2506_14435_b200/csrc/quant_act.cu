@@ -120,7 +120,7 @@ __global__ void __launch_bounds__(256) quant_act_kernel(QuantActArgs a) {
           const bool m = pp < pair && a.topk_idx[pp] == e;
           rank += __popc(__ballot_sync(0xffffffffu, m));
         }
-        dst = a.blk_base[blk * a.E + e] + rank;
+        dst = a.blk_base[e * blk_stride(a.n_blk) + blk] + rank;
         if (tg == 0) {
           a.perm_out[pair] = (int32_t)dst;
           a.inv_out[dst] = pair;

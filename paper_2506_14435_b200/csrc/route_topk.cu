@@ -286,7 +286,7 @@ __global__ void __launch_bounds__(kRmWarps * 32) route_topk_mma_kernel(const uin
   }
   if (blk_hist) {                                      // input of the block-wise dispatch (dispatch.cu)
     __syncthreads();
-    if (threadIdx.x < E) blk_hist[int64_t(blockIdx.x) * E + threadIdx.x] = s_hist[threadIdx.x];
+    if (threadIdx.x < E) blk_hist[int64_t(threadIdx.x) * blk_stride((int)gridDim.x) + blockIdx.x] = s_hist[threadIdx.x];
   }
 }
 
