@@ -18,7 +18,7 @@
 namespace mote {
 
 template <int kUnits, bool kScatter>
-__global__ void __launch_bounds__(256) quant_act_kernel(QuantActArgs a) {
+__global__ void __launch_bounds__(256, kUnits <= 2 ? 4 : 1) quant_act_kernel(QuantActArgs a) {
   __shared__ float s_max[8];
   __shared__ int s_sum[8];
   const int G = a.group;                          // threads per row
@@ -381,9 +381,10 @@ mote_status_t launch_quant_act(const QuantActArgs& a, bool scatter, cudaStream_t
     return MOTE_OK;
   }
   const int n_units = a.d / 16;
-  // smallest power-of-two group with at most 4 units per thread (8 for the widest rows)
+  // smallest power-of-two group with at most 2 units per thread (up to 8 for the widest rows): with
+  // two the kernel fits four CTAs per SM, and it is the rows in flight per SM that set its time
   int G = 32;
-  while (G < 256 && n_units > G * 4) G <<= 1;
+  while (G < 256 && n_units > G * 2) G <<= 1;
   const int upt = (n_units + G - 1) / G;
   QuantActArgs args = a;
   args.group = G;
