@@ -230,8 +230,8 @@ __global__ void __launch_bounds__(256, 4) quant_act_rows_kernel(QuantActArgs a) 
 // half-integer: |r - 127x/beta| <= 127 * 3 * 2^-24 and |fl(fl(127x)/beta) - 127x/beta| <= 127 * 2^-24
 // add up to 3.03e-5 < 2^-14, so outside that band both round to the same integer.  A unit with such
 // an element (one in 500) is redone by an out-of-line function, so that the streaming loop holds
-// neither the division's instructions nor a branch per element: 9.4 instead of 20 instructions per
-// element.  (The two kernels above keep the branch per element: with the out-of-line call the
+// neither the division's instructions nor a branch per element: 13 instead of 18 instructions per
+// element on rows of 4864, 9.4 on rows of 11008.  (The two kernels above keep the branch per element: with the out-of-line call the
 // row-staging kernel spills and drops from 3.5 to 2.9 TB/s, and the scatter kernel gains at
 // T = 8192 what it loses at T <= 4096, under 0.4 % of the layer either way.)
 constexpr float kQaFastBand = 0.49993896484375f;   // 0.5 - 2^-14
