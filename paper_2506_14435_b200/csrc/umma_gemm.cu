@@ -60,6 +60,7 @@ struct UmmaArgs {
   int k_splits;             // down projections: items per output tile, each over 1/k_splits of K (>= 1)
   int64_t split_stride;     // elements between the partial outputs of consecutive splits
   int bn;                   // weight rows per tile (UMMA N)
+  int split_tail;           // down projections with bn = 256, k_splits = 1: see plan_items
   int n_out;                // output row length (f for gate/up, d for down)
   int b_rows_per_expert;    // rows of the weight tensor map per expert (0: shared expert)
   const float* beta;        // [rows]   (ternary modes)
@@ -116,8 +117,33 @@ struct ModeTraits {
 //            L2 for long prefills), which is then read from HBM once instead of once per column tile.
 // A down projection with few row tiles may split K over k_splits items per output tile (each
 // writes its partial sums; the caller adds them in a fixed order): item = (row tile, split, column tile).
+//
+// The items of the last, partial round of the persistent grid would leave most SMs idle for a whole
+// tile time (512 tiles on 148 CTAs: 3.46 rounds cost 4).  Where at most half of the CTAs have a
+// tile left in that round, a down projection with 256-column tiles cuts each of those tiles into its
+// two 128-column halves, one item each: the round then takes 0.57 of a tile time (the MMA pipe runs
+// N = 128 at 0.87 of its N = 256 rate).  Items [0, n_whole) are whole tiles, [n_whole, n_items) halves.
+struct ItemPlan { int n_items, n_whole; };
 template <bool kGateUp>
-__device__ __forceinline__ void decode_item(const UmmaArgs& a, int item, int n_mtiles, int4& tile, int& n_tile) {
+__device__ __forceinline__ ItemPlan plan_items(const UmmaArgs& a, int n_mtiles) {
+  ItemPlan p;
+  p.n_items = p.n_whole = n_mtiles * a.n_ntiles * (kGateUp ? 1 : a.k_splits);
+  if (!kGateUp && a.split_tail) {
+    const int tail = p.n_items % (int)gridDim.x;
+    if (tail > 0 && 2 * tail <= (int)gridDim.x) { p.n_whole = p.n_items - tail; p.n_items += tail; }
+  }
+  return p;
+}
+// half: -1 for a whole tile, else which 128-column half of tile (m_tile, n_tile) the item is
+template <bool kGateUp>
+__device__ __forceinline__ void decode_item(const UmmaArgs& a, int item, int n_mtiles, int n_whole, int4& tile,
+                                            int& n_tile, int& half) {
+  half = -1;
+  if (!kGateUp && item >= n_whole) {
+    const int j = item - n_whole;
+    item = n_whole + (j >> 1);
+    half = j & 1;
+  }
   int m_tile;
   if (kGateUp) { m_tile = item % n_mtiles; n_tile = item / n_mtiles; }
   else { m_tile = item / (a.n_ntiles * a.k_splits); n_tile = item % a.n_ntiles; }
@@ -203,7 +229,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
   const uint32_t tmem_base = bars->tmem_base;
   pdl_wait();                              // set-up above overlaps the tail of the kernel before this one
   const int n_mtiles = a.tiles[0].x;
-  const int n_items = n_mtiles * a.n_ntiles * (TR::kGateUp ? 1 : a.k_splits);
+  const ItemPlan plan = plan_items<TR::kGateUp>(a, n_mtiles);
+  const int n_items = plan.n_items, n_whole = plan.n_whole;
 
   if (warp == 0) {
     // ---------------------------------------------------------------- token-operand producer
@@ -211,9 +238,11 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
       uint32_t stage = 0, phase = 0;
       bool ok = true;
       for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x) {
-        int4 tile; int n_tile;
-        decode_item<TR::kGateUp>(a, item, n_mtiles, tile, n_tile);
-        const int b_row = (a.b_rows_per_expert ? tile.x * a.b_rows_per_expert : 0) + n_tile * (TR::kGateUp ? a.bn / 2 : a.bn);
+        int4 tile; int n_tile, half;
+        decode_item<TR::kGateUp>(a, item, n_mtiles, n_whole, tile, n_tile, half);
+        const int width = half < 0 ? a.bn : 128;
+        const int b_row = (a.b_rows_per_expert ? tile.x * a.b_rows_per_expert : 0) +
+                          n_tile * (TR::kGateUp ? a.bn / 2 : a.bn) + (half > 0 ? 128 : 0);
         int kb, ke;
         item_k_range<TR::kGateUp>(a, item, kb, ke);
         for (int ks = kb; ks < ke; ++ks) {
@@ -226,14 +255,14 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
             mbar_expect_tx(bar, kStageA);
             tma_load_2d(sA + stage * kStageA, &tm_a, ks * 64, tile.y, bar);
           } else {
-            mbar_expect_tx(bar, kStageA + a.bn * 128);
+            mbar_expect_tx(bar, kStageA + width * 128);
             tma_load_2d(sA + stage * kStageA, &tm_a, ks * 64, tile.y, bar);
             if (TR::kGateUp) {
               tma_load_2d(sB + stage * kStageB, &tm_b0, ks * 64, b_row, bar);
               tma_load_2d(sB + stage * kStageB + 128 * 128, &tm_b1, ks * 64, b_row, bar);
             } else {
               tma_load_2d(sB + stage * kStageB, &tm_b0, ks * 64, b_row, bar);
-              if (a.bn > 128) tma_load_2d(sB + stage * kStageB + 128 * 128, &tm_b1, ks * 64, b_row + 128, bar);
+              if (width > 128) tma_load_2d(sB + stage * kStageB + 128 * 128, &tm_b1, ks * 64, b_row + 128, bar);
             }
           }
           if (++stage == S) { stage = 0; phase ^= 1; }
@@ -247,22 +276,23 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
       uint32_t stage = 0, phase = 0;
       bool ok = true;
       for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x) {
-        int4 tile; int n_tile;
-        decode_item<TR::kGateUp>(a, item, n_mtiles, tile, n_tile);
-        const int b_row = tile.x * a.b_rows_per_expert + n_tile * (TR::kGateUp ? a.bn / 2 : a.bn);
+        int4 tile; int n_tile, half;
+        decode_item<TR::kGateUp>(a, item, n_mtiles, n_whole, tile, n_tile, half);
+        const int width = half < 0 ? a.bn : 128;
+        const int b_row = tile.x * a.b_rows_per_expert + n_tile * (TR::kGateUp ? a.bn / 2 : a.bn) + (half > 0 ? 128 : 0);
         int kb, ke;
         item_k_range<TR::kGateUp>(a, item, kb, ke);
         for (int ks = kb; ks < ke; ++ks) {
           if (!(ok = mbar_wait(smem_u32(&bars->empty_p[stage]), phase ^ 1, abort_flag))) break;
           const uint32_t bar = smem_u32(&bars->full_p[stage]);
-          mbar_expect_tx(bar, a.bn * kRB);
+          mbar_expect_tx(bar, width * kRB);
           const uint32_t dst = sP + stage * TR::kStageP;
           if (TR::kGateUp) {
             tma_load_2d(dst, &tm_b0, ks * kRB, b_row, bar);
             tma_load_2d(dst + 128 * kRB, &tm_b1, ks * kRB, b_row, bar);
           } else {
             tma_load_2d(dst, &tm_b0, ks * kRB, b_row, bar);
-            if (a.bn > 128) tma_load_2d(dst + 128 * kRB, &tm_b1, ks * kRB, b_row + 128, bar);
+            if (width > 128) tma_load_2d(dst + 128 * kRB, &tm_b1, ks * kRB, b_row + 128, bar);
           }
           if (++stage == TR::kStagesP) { stage = 0; phase ^= 1; }
         }
@@ -271,8 +301,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
   } else if (warp == 2) {
     // ---------------------------------------------------------------- MMA issuer
     if (lane == 0) {
-      const uint32_t idesc = TR::kTernary ? make_idesc(2, 1, 0, kBM, (uint32_t)a.bn)     // s32 += s8 * u8
-                                          : make_idesc(1, 1, 1, kBM, (uint32_t)a.bn);    // f32 += bf16 * bf16
+      const uint32_t idesc_whole = TR::kTernary ? make_idesc(2, 1, 0, kBM, (uint32_t)a.bn)     // s32 += s8 * u8
+                                                : make_idesc(1, 1, 1, kBM, (uint32_t)a.bn);    // f32 += bf16 * bf16
+      const uint32_t idesc_half = TR::kTernary ? make_idesc(2, 1, 0, kBM, 128u) : make_idesc(1, 1, 1, kBM, 128u);
       uint32_t stage = 0, phase = 0;
       int local = 0;
       bool ok = true;
@@ -282,6 +313,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
         if (!(ok = mbar_wait(smem_u32(&bars->tmem_empty[buf]), (use & 1) ^ 1, abort_flag))) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * 256;
+        const uint32_t idesc = (!TR::kGateUp && item >= n_whole) ? idesc_half : idesc_whole;
         int kb, ke;
         item_k_range<TR::kGateUp>(a, item, kb, ke);
         for (int ks = kb; ks < ke; ++ks) {
@@ -312,8 +344,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
       const int tid = (threadIdx.x - 128) & 127;
       uint32_t stage = 0, phase = 0, pstage = 0, pphase = 0, step = 0;
       bool ok = true;
-      const int n_chunks = a.bn * (TR::kCodeRowBytes / 16);   // chunks of 16 code bytes, spread over 128 threads
       for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x) {
+        // chunks of 16 code bytes, spread over 128 threads
+        const int n_chunks = ((!TR::kGateUp && item >= n_whole) ? 128 : a.bn) * (TR::kCodeRowBytes / 16);
         int kb, ke;
         item_k_range<TR::kGateUp>(a, item, kb, ke);
         for (int ks = kb; ks < ke; ++ks, ++step) {
@@ -388,8 +421,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
     int local = 0;
     bool ok = true;
     for (int item = blockIdx.x; ok && item < n_items; item += gridDim.x, ++local) {
-      int4 tile; int n_tile;
-      decode_item<TR::kGateUp>(a, item, n_mtiles, tile, n_tile);
+      int4 tile; int n_tile, half;
+      decode_item<TR::kGateUp>(a, item, n_mtiles, n_whole, tile, n_tile, half);
       int kb_, ke_;
       const int split = item_k_range<TR::kGateUp>(a, item, kb_, ke_);
       const int buf = local & 1;
@@ -508,8 +541,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
           if (hb) atomicMax(a.beta_out_bits + row, hb);
         }
       } else {
-        const int col0 = n_tile * a.bn;
-        const int cbeg = chalf * (a.bn / 2), cend = cbeg + a.bn / 2;
+        const int width = half < 0 ? a.bn : 128;
+        const int col0 = n_tile * a.bn + (half > 0 ? 128 : 0);
+        const int cbeg = chalf * (width / 2), cend = cbeg + width / 2;
         const bool combine = !TR::kTernary && a.comb_out != nullptr;
         float cw[MOTE_MAX_TOPK];
         const float* cy[MOTE_MAX_TOPK];
@@ -720,6 +754,7 @@ mote_status_t launch_ternary_umma(const TernaryGemmArgs& g, bool gateup, const i
   a.k_steps = g.K / 128;
   a.k_splits = 1;
   a.bn = bn;
+  a.split_tail = (!gateup && bn == 256) ? 1 : 0;
   a.n_out = g.N;
   a.b_rows_per_expert = g.N;
   a.beta = g.beta; a.rowsum = rowsum; a.alpha0 = g.alpha0; a.alpha1 = g.alpha1;
@@ -781,6 +816,7 @@ mote_status_t launch_shared_umma(const void* act, const SharedMat& w0, const Sha
   a.k_splits = std::max(k_splits, 1);
   a.split_stride = T * N;
   a.bn = bn;
+  a.split_tail = (!gateup && bn == 256 && a.k_splits == 1) ? 1 : 0;
   a.n_out = N;
   a.b_rows_per_expert = 0;
   a.out = out;
