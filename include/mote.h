@@ -262,7 +262,13 @@ mote_status_t mote_moe_forward(const mote_layer_t* L, const void* x_bf16,
 /* Same layer with HOST input and output: copies x_host (and residual_host if non-NULL) to the
  * device, runs mote_moe_forward, copies the result to out_host and waits for the stream.  Host
  * buffers should be page-locked for the copies to be asynchronous.  Needs
- * mote_layer_workspace_bytes(...) + mote_host_staging_bytes(d, T) bytes of device scratch. */
+ * mote_layer_workspace_bytes(...) + mote_host_staging_bytes(d, T) bytes of device scratch.
+ * From 4096 tokens on the call runs the layer as two halves of the tokens (Eq. 2-4 treat every
+ * token on its own, so the result is bit-identical to the one-piece call): the second half's input
+ * copy runs beside the first half's layer and the first half's output copy beside the second
+ * half's layer, on two copy streams that the library creates on the calling thread's first such
+ * call on a device and keeps.  The copies start after the work already queued on `stream`; when
+ * the call returns, `stream` and both copy streams are idle. */
 size_t mote_host_staging_bytes(int d, int64_t T_max);
 mote_status_t mote_moe_forward_host(const mote_layer_t* L, const void* x_host,
                                     const void* residual_host, int64_t T, void* out_host,

@@ -532,6 +532,34 @@ extern "C" mote_status_t mote_stack_forward(const mote_layer_t* layers, int n_la
   return MOTE_OK;
 }
 
+// Copy streams and events of the pipelined host call below: made on a thread's first long call on a
+// device and kept for the thread's life time.
+struct HostPipe {
+  cudaStream_t in = nullptr, out = nullptr;
+  cudaEvent_t start = nullptr, copied[2] = {nullptr, nullptr}, computed[2] = {nullptr, nullptr}, done = nullptr;
+  bool ready = false;
+};
+static thread_local HostPipe g_host_pipe[kMaxDevices];
+
+static HostPipe* host_pipe() {
+  const int dev = current_device();
+  if (dev < 0 || dev >= kMaxDevices) return nullptr;
+  HostPipe& p = g_host_pipe[dev];
+  if (p.ready) return &p;
+  bool ok = cudaStreamCreateWithFlags(&p.in, cudaStreamNonBlocking) == cudaSuccess &&
+            cudaStreamCreateWithFlags(&p.out, cudaStreamNonBlocking) == cudaSuccess;
+  cudaEvent_t* evs[] = {&p.start, &p.copied[0], &p.copied[1], &p.computed[0], &p.computed[1], &p.done};
+  for (cudaEvent_t* e : evs) ok = ok && cudaEventCreateWithFlags(e, cudaEventDisableTiming) == cudaSuccess;
+  if (!ok) return nullptr;                             // the caller falls back to the plain sequence
+  p.ready = true;
+  return &p;
+}
+
+// Prefills of this many tokens or more go through the device as two halves: the second half's input
+// copy runs beside the first half's layer, the first half's output copy beside the second half's
+// layer (tokens are independent of one another, Eq. 2-4, so the halves are too).
+constexpr int64_t kHostPipelineMinTokens = 4096;
+
 extern "C" mote_status_t mote_moe_forward_host(const mote_layer_t* L, const void* x_host, const void* residual_host,
                                                int64_t T, void* out_host, void* ws, size_t ws_bytes, void* stream_) {
   if (!L) return MOTE_ERR_NULL;
@@ -544,17 +572,57 @@ extern "C" mote_status_t mote_moe_forward_host(const mote_layer_t* L, const void
   if (ws_bytes < core + 3 * slab) return MOTE_ERR_WORKSPACE;
   cudaStream_t stream = static_cast<cudaStream_t>(stream_);
   char* stage = static_cast<char*>(ws) + core;
-  void* x_dev = stage;
-  void* res_dev = residual_host ? stage + slab : nullptr;
-  void* out_dev = stage + 2 * slab;
-  const size_t bytes = size_t(T) * L->d * 2;
-  MOTE_CUDA_OK(cudaMemcpyAsync(x_dev, x_host, bytes, cudaMemcpyHostToDevice, stream));
-  if (residual_host) MOTE_CUDA_OK(cudaMemcpyAsync(res_dev, residual_host, bytes, cudaMemcpyHostToDevice, stream));
-  mote_status_t st = mote_moe_forward(L, x_dev, res_dev, T, out_dev, nullptr, ws, core, stream);
+  char* x_dev = stage;
+  char* res_dev = residual_host ? stage + slab : nullptr;
+  char* out_dev = stage + 2 * slab;
+  const size_t row = size_t(L->d) * 2;
+  const size_t bytes = size_t(T) * row;
+  HostPipe* pipe = T >= kHostPipelineMinTokens ? host_pipe() : nullptr;
+  if (!pipe) {
+    MOTE_CUDA_OK(cudaMemcpyAsync(x_dev, x_host, bytes, cudaMemcpyHostToDevice, stream));
+    if (residual_host) MOTE_CUDA_OK(cudaMemcpyAsync(res_dev, residual_host, bytes, cudaMemcpyHostToDevice, stream));
+    mote_status_t st = mote_moe_forward(L, x_dev, res_dev, T, out_dev, nullptr, ws, core, stream);
+    if (st) return st;
+    MOTE_CUDA_OK(cudaMemcpyAsync(out_host, out_dev, bytes, cudaMemcpyDeviceToHost, stream));
+    MOTE_CUDA_OK(cudaStreamSynchronize(stream));
+    return MOTE_OK;
+  }
+  const int64_t t0[3] = {0, (T / 2 + 127) / 128 * 128, T};       // the halves: whole row tiles in the first
+  MOTE_CUDA_OK(cudaEventRecord(pipe->start, stream));             // the copies start after the stream's earlier work
+  MOTE_CUDA_OK(cudaStreamWaitEvent(pipe->in, pipe->start, 0));
+  for (int c = 0; c < 2; ++c) {
+    const size_t off = size_t(t0[c]) * row, n = size_t(t0[c + 1] - t0[c]) * row;
+    MOTE_CUDA_OK(cudaMemcpyAsync(x_dev + off, static_cast<const char*>(x_host) + off, n, cudaMemcpyHostToDevice, pipe->in));
+    if (residual_host)
+      MOTE_CUDA_OK(cudaMemcpyAsync(res_dev + off, static_cast<const char*>(residual_host) + off, n, cudaMemcpyHostToDevice,
+                                   pipe->in));
+    MOTE_CUDA_OK(cudaEventRecord(pipe->copied[c], pipe->in));
+  }
+  MOTE_CUDA_OK(cudaMemsetAsync(ws, 0, 4, stream));                // device status word: once for both halves
+  mote_status_t st = MOTE_OK;
+  {
+    struct KeepStatus { KeepStatus() { g_keep_status = true; } ~KeepStatus() { g_keep_status = false; } } keep_status;
+    for (int c = 0; c < 2 && st == MOTE_OK; ++c) {
+      const size_t off = size_t(t0[c]) * row;
+      if (cudaStreamWaitEvent(stream, pipe->copied[c], 0) != cudaSuccess) { st = MOTE_ERR_CUDA; break; }
+      st = mote_moe_forward(L, x_dev + off, res_dev ? res_dev + off : nullptr, t0[c + 1] - t0[c], out_dev + off, nullptr,
+                            ws, core, stream);
+      if (st) break;
+      if (cudaEventRecord(pipe->computed[c], stream) != cudaSuccess ||
+          cudaStreamWaitEvent(pipe->out, pipe->computed[c], 0) != cudaSuccess ||
+          cudaMemcpyAsync(static_cast<char*>(out_host) + off, out_dev + off, size_t(t0[c + 1] - t0[c]) * row,
+                          cudaMemcpyDeviceToHost, pipe->out) != cudaSuccess)
+        st = MOTE_ERR_CUDA;
+    }
+  }
+  // whatever happened, leave none of the helper streams' work behind
+  const bool drained = cudaEventRecord(pipe->done, pipe->out) == cudaSuccess &&
+                       cudaStreamWaitEvent(stream, pipe->done, 0) == cudaSuccess;
+  const bool in_ok = cudaStreamSynchronize(pipe->in) == cudaSuccess;
+  const bool out_ok = cudaStreamSynchronize(pipe->out) == cudaSuccess;
+  const bool main_ok = cudaStreamSynchronize(stream) == cudaSuccess;
   if (st) return st;
-  MOTE_CUDA_OK(cudaMemcpyAsync(out_host, out_dev, bytes, cudaMemcpyDeviceToHost, stream));
-  MOTE_CUDA_OK(cudaStreamSynchronize(stream));
-  return MOTE_OK;
+  return (drained && in_ok && out_ok && main_ok) ? MOTE_OK : MOTE_ERR_CUDA;
 }
 
 extern "C" mote_status_t mote_moe_forward_profile(const mote_layer_t* L, const void* x, const void* residual,

@@ -165,6 +165,26 @@ def test_host_buffer_entry_point(mote):
     assert torch.equal(out_host, want.cpu())
 
 
+@pytest.mark.parametrize("T,with_residual", [(4096, False), (4133, True), (9000, True)])
+def test_host_buffer_entry_point_long_prefill(mote, T, with_residual):
+    """From 4096 tokens on the host call runs the layer as two halves with the copies of one half
+    beside the layer of the other: the result must equal the one-piece device call bit for bit
+    (tokens are independent, Eq. 2-4), for an even and for a ragged split.  (The device call is
+    what the other tests compare with the oracle.)"""
+    from paper_2506_14435_b200.binding import mote_moe_forward_host
+    wl = synth.Workload("host_pipe", 128, 256, 8, 2, T, seed=77, bias="zipf")
+    master, layer_or, layer_gpu = _setup(mote, wl)
+    pin = lambda bits: torch.from_numpy(bits.view(np.int16).copy()).view(torch.bfloat16).pin_memory()
+    x_host = pin(synth.tokens(wl))
+    res_host = pin(synth.tokens(wl, stream=1)) if with_residual else None
+    out_host = torch.empty_like(x_host).pin_memory()
+    for _ in range(2):                                   # the second call reuses the copy streams
+        out_host.zero_()
+        mote_moe_forward_host(layer_gpu, x_host, out_host, res_host)
+        want = mote.mote_moe_forward(layer_gpu, x_host.cuda(), residual=None if res_host is None else res_host.cuda())
+        assert torch.equal(out_host, want.cpu())
+
+
 # ------------------------------------------------------------------ Section 4.3: RTN-coded shared expert
 @pytest.mark.parametrize("bits", [8, 4])
 @pytest.mark.parametrize("d,f,E,k,T,kw,path", [
