@@ -445,6 +445,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
       if (TR::kGateUp) {
         const int col0 = n_tile * 128;
         const bool row_fast = __fmul_rn(c0, c1) > 1e-12f;
+        const uint32_t acc_bias = 0x4B400000u - (uint32_t)rs;
         float hmax = 0.0f;                           // max |h| (before the bf16 rounding, which is monotonic)
         constexpr int kCols = TR::kEpiCols, kPitch = TR::kEpiPitch;
         constexpr int kLanesPerRow = kCols * 2 / 16, kRowsPerStore = 32 / kLanesPerRow;
@@ -464,14 +465,18 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
 #pragma unroll
                 for (int j = 0; j < 16; ++j) {
                   bool redo;
-                  hv[j] = glu_h_fast((int)rg[j] - rs, (int)ru[j] - rs, c0, c1, redo);
+                  hv[j] = glu_h_fast_biased(rg[j], ru[j], acc_bias, c0, c1, redo);
                   if (redo) redo_mask |= 1u << j;
                 }
                 if (!row_fast) redo_mask = 0xFFFFu;
-                if (redo_mask) {
+                if (redo_mask) {                     // mostly one element: look at four at a time
 #pragma unroll
-                  for (int j = 0; j < 16; ++j)
-                    if ((redo_mask >> j) & 1u) hv[j] = glu_h_rare((int)rg[j] - rs, (int)ru[j] - rs, c0, c1);
+                  for (int j0 = 0; j0 < 16; j0 += 4)
+                    if ((redo_mask >> j0) & 0xFu) {
+#pragma unroll
+                      for (int j = j0; j < j0 + 4; ++j)
+                        if ((redo_mask >> j) & 1u) hv[j] = glu_h_rare((int)rg[j] - rs, (int)ru[j] - rs, c0, c1);
+                    }
                 }
 #pragma unroll
                 for (int j = 0; j < 16; ++j) hmax = fmaxf(hmax, fabsf(hv[j]));
@@ -541,6 +546,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
           if (hb) atomicMax(a.beta_out_bits + row, hb);
         }
       } else {
+        const uint32_t acc_bias = 0x4B400000u - (uint32_t)rs;   // see glu_h_fast_biased
         const int width = half < 0 ? a.bn : 128;
         const int col0 = n_tile * a.bn + (half > 0 ? 128 : 0);
         const int cbeg = chalf * (width / 2), cend = cbeg + width / 2;
@@ -564,7 +570,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tm_a, const __grid_constant
             float o[16];
 #pragma unroll
             for (int v = 0; v < 16; ++v)
-              o[v] = TR::kTernary ? __fmul_rn(i2f_small((int)ra[v] - rs), c0) : __uint_as_float(ra[v]);
+              o[v] = TR::kTernary ? __fmul_rn(__fsub_rn(__uint_as_float(ra[v] + acc_bias), kMagic), c0)   // fl32(acc - rs) * c0
+                                  : __uint_as_float(ra[v]);
             if (TR::kRtn || (!TR::kTernary && a.alpha0 != nullptr)) {
               const float4* sp = reinterpret_cast<const float4*>(a.alpha0 + col0 + c);
 #pragma unroll
