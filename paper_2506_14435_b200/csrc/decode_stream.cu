@@ -89,7 +89,6 @@ __global__ void __launch_bounds__(256) decode_prologue_kernel(DecodePrologueArgs
   const int t = blockIdx.x;
   const int d = a.d, n_vec = d / 8, n_units = d / 16;
   const uint4* src = reinterpret_cast<const uint4*>(a.x + int64_t(t) * d);
-  pdl_trigger();                         // the gate/up kernel may start on the shared expert right away
 
   // The router weights do not depend on the token: the first pass's rows for this thread's first
   // unit are requested now, and the later passes' rows are pulled into L2, so that their latency
@@ -104,6 +103,11 @@ __global__ void __launch_bounds__(256) decode_prologue_kernel(DecodePrologueArgs
     for (int e = 8; e < a.E; ++e)
       asm volatile("prefetch.global.L2 [%0];" ::"l"(a.Wr + int64_t(e) * d + 8 * tid));
   }
+  // x may be the output of the kernel ahead (the RMS norm of a layer stack, launched as this kernel's
+  // programmatic predecessor).  Only then may the gate/up kernel start on the shared expert, which
+  // reads x too.
+  pdl_wait();
+  pdl_trigger();
 
   float amax = 0.0f;
   for (int v = tid; v < n_vec; v += 256) {
@@ -946,7 +950,7 @@ mote_status_t launch_decode_stream(const DecodeStreamArgs& p, int phase, cudaStr
     pa.rowsum_h = p.rowsum_h; pa.counter = p.counter; pa.offsets = p.offsets; pa.perm = p.perm; pa.inv = p.inv;
     static PerDeviceOnce prologue_attr;
     MOTE_CUDA_OK(set_max_dynamic_smem(prologue_attr, decode_prologue_kernel, 32768));
-    decode_prologue_kernel<<<T, 256, size_t(d) * 2, stream>>>(pa);
+    MOTE_CUDA_OK(launch_pdl(decode_prologue_kernel, dim3(T), dim3(256), size_t(d) * 2, stream, pa));
     ++g_launch_count;
     MOTE_LAUNCH_OK();
     return MOTE_OK;

@@ -17,6 +17,10 @@ thread_local int g_launch_count = 0;
 // out in ANY layer is still there when the caller reads mote_device_status after the stack.
 static thread_local bool g_keep_status = false;
 
+// Head of a workspace: the status word, the decode prologue's arrival counter and the decode down
+// kernel's tile counters (one per 16 output columns, from byte 256 on).
+static inline size_t status_region_bytes(int d) { return 256 + size_t(d / 16) * 4; }
+
 // Optional per-stage CUDA events (mote_moe_forward_profile): event i is recorded on the launch
 // stream after stage i has been enqueued, event 0 before the first stage.
 struct StageTimer {
@@ -287,8 +291,8 @@ extern "C" mote_status_t mote_moe_forward(const mote_layer_t* L, const void* x, 
 
   if (path == MOTE_PATH_STREAM) {
     // status word, the prologue's arrival counter, the down kernel's tile counters
-    const size_t keep = g_keep_status ? 4 : 0;
-    MOTE_CUDA_OK(cudaMemsetAsync(reinterpret_cast<char*>(status) + keep, 0, 256 + size_t(d / 16) * 4 - keep, stream));
+    // (the kernels leave their counters at zero, so inside a stack the stack's one memset is enough)
+    if (!g_keep_status) MOTE_CUDA_OK(cudaMemsetAsync(status, 0, status_region_bytes(d), stream));
     stage_mark(0, stream);
     DecodeStreamArgs ds{};
     ds.x = x; ds.T = T; ds.d = d; ds.f = f; ds.E = E; ds.k = k; ds.norm_topk = L->norm_topk;
@@ -508,7 +512,8 @@ extern "C" mote_status_t mote_stack_forward(const mote_layer_t* layers, int n_la
   void* normed = ping + 2 * slab;
   int launches = 0;
   const void* res = x;                                 // residual stream x_{l-1}
-  MOTE_CUDA_OK(cudaMemsetAsync(ws, 0, 4, stream));     // device status word: once for the whole stack
+  // device status word and the decode kernels' counters: once for the whole stack
+  MOTE_CUDA_OK(cudaMemsetAsync(ws, 0, status_region_bytes(d), stream));
   struct KeepStatus { KeepStatus() { g_keep_status = true; } ~KeepStatus() { g_keep_status = false; } } keep_status;
   for (int l = 0; l < n_layers; ++l) {
     void* dst = (l == n_layers - 1) ? out : static_cast<void*>(ping + size_t(l & 1) * slab);
@@ -598,7 +603,7 @@ extern "C" mote_status_t mote_moe_forward_host(const mote_layer_t* L, const void
                                    pipe->in));
     MOTE_CUDA_OK(cudaEventRecord(pipe->copied[c], pipe->in));
   }
-  MOTE_CUDA_OK(cudaMemsetAsync(ws, 0, 4, stream));                // device status word: once for both halves
+  MOTE_CUDA_OK(cudaMemsetAsync(ws, 0, status_region_bytes(L->d), stream));   // status word, counters: once for both halves
   mote_status_t st = MOTE_OK;
   {
     struct KeepStatus { KeepStatus() { g_keep_status = true; } ~KeepStatus() { g_keep_status = false; } } keep_status;

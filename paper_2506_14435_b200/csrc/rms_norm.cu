@@ -12,6 +12,7 @@ __global__ void __launch_bounds__(256) rms_norm_kernel(const uint16_t* __restric
                                                        uint16_t* __restrict__ y) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int64_t row = int64_t(blockIdx.x) * 8 + warp;
+  pdl_wait();                            // x may be the output of the kernel ahead (a layer stack)
   if (row >= T) return;
   const uint4* src = reinterpret_cast<const uint4*>(x + row * int64_t(d));
   uint4* dst = reinterpret_cast<uint4*>(y + row * int64_t(d));
@@ -41,8 +42,8 @@ __global__ void __launch_bounds__(256) rms_norm_kernel(const uint16_t* __restric
 
 mote_status_t launch_rms_norm(const void* x, int64_t T, int d, float eps, void* y, cudaStream_t stream) {
   if (T == 0) return MOTE_OK;
-  rms_norm_kernel<<<(unsigned)((T + 7) / 8), 256, 0, stream>>>(static_cast<const uint16_t*>(x), T, d, eps,
-                                                            static_cast<uint16_t*>(y));
+  MOTE_CUDA_OK(launch_pdl(rms_norm_kernel, dim3((unsigned)((T + 7) / 8)), dim3(256), 0, stream,
+                          static_cast<const uint16_t*>(x), T, d, eps, static_cast<uint16_t*>(y)));
   ++g_launch_count;
   MOTE_LAUNCH_OK();
   return MOTE_OK;
