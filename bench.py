@@ -66,12 +66,15 @@ def measured_peaks():
 
 
 class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples SM clocks and throttle reasons with nvidia-smi (every 20 ms) and reports the samples
+    that fall between begin() and end(): start it early enough (wait_first) that the tool is already
+    printing when the timed region begins."""
     FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
               "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
     def __init__(self, index: int):
         self.index, self.proc, self.lines = index, None, []
+        self.t_begin = self.t_end = None
 
     def start(self):
         try:
@@ -86,29 +89,51 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.lines.append(line.strip())
+            self.lines.append((time.monotonic(), line.strip()))
+
+    def wait_first(self, timeout: float = 1.0):
+        """Returns once the first sample has arrived (or after `timeout` seconds)."""
+        t0 = time.monotonic()
+        while self.proc is not None and not self.lines and time.monotonic() - t0 < timeout:
+            time.sleep(0.005)
+        return self
+
+    def begin(self):
+        self.t_begin = time.monotonic()
+
+    def end(self):
+        self.t_end = time.monotonic()
 
     def stop(self) -> dict:
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.12)
+        if self.t_end is None:
+            self.end()
+        time.sleep(0.045)                               # the sample that was being taken when the region ended
         self.proc.terminate()
         self.thread.join(timeout=2)
-        sm, mx, reasons = [], None, set()
+        parsed = []
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for ln in self.lines:
+        for t, ln in self.lines:
             p = [s.strip() for s in ln.split(",")]
             if len(p) < 6:
                 continue
             try:
-                sm.append(float(p[0])); mx = float(p[1])
+                parsed.append((t, float(p[0]), float(p[1]),
+                               [n for n, v in zip(names, p[2:6]) if v.lower().startswith("active")]))
             except ValueError:
                 continue
-            for n, v in zip(names, p[2:6]):
-                if v.lower().startswith("active"):
-                    reasons.add(n)
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": mx, "reasons": sorted(reasons),
-                "samples": len(sm)}
+        # a line is read within a few ms of its sample; samples of the region, else the one nearest to it
+        lo = (self.t_begin if self.t_begin is not None else 0.0) + 0.002
+        hi = self.t_end + 0.022
+        inside = [q for q in parsed if lo <= q[0] <= hi]
+        if not inside and parsed:
+            mid = 0.5 * (lo + hi)
+            inside = [min(parsed, key=lambda q: abs(q[0] - mid))]
+        sm = [q[1] for q in inside]
+        reasons = sorted({r for q in inside for r in q[3]})
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": inside[-1][2] if inside else None,
+                "reasons": reasons, "samples": len(sm)}
 
 
 def stage_work(wl: synth.Workload, stage: str, stream_path: bool, experts_touched: float, shared_bits: int = 16,
@@ -183,7 +208,9 @@ def int8_peak(mote_binding, rank: int, local_rank: int) -> dict:
     a few 5 ms launches from idle clocks) and a sustained one (median launch of the second half of
     about a second of back-to-back launches, clocks sampled meanwhile)."""
     burst = mote_binding.mote_int8_mma_peak(800, repeats=5)
-    sampler = ClockSampler(local_rank).start() if rank == 0 else None
+    sampler = ClockSampler(local_rank).start().wait_first() if rank == 0 else None
+    if sampler:
+        sampler.begin()
     long = mote_binding.mote_int8_mma_peak(1600, repeats=80)
     clocks = sampler.stop() if sampler else None
     ms = long["ms_in_order"][len(long["ms_in_order"]) // 2:]
@@ -303,8 +330,10 @@ def measure(ls: LayerSet, wl: synth.Workload, args, steps: int | None, rank: int
         step_timed = graph.replay
         for _ in range(3):
             step_timed()
+    sampler = ClockSampler(local_rank).start().wait_first() if rank == 0 else None
     barrier()
-    sampler = ClockSampler(local_rank).start() if rank == 0 else None
+    if sampler:
+        sampler.begin()
     per_step = timed_loop(step_timed, steps)
     barrier()
     clocks = sampler.stop() if sampler else None
@@ -314,7 +343,9 @@ def measure(ls: LayerSet, wl: synth.Workload, args, steps: int | None, rank: int
     # loop about as long as the timed one, so that both run at the same clocks
     stage_acc = {}
     n_prof = max(3, min(steps, int(500.0 / max(total_ms / steps, 1e-3)) + 1))
-    sampler = ClockSampler(local_rank).start() if rank == 0 else None
+    sampler = ClockSampler(local_rank).start().wait_first() if rank == 0 else None
+    if sampler:
+        sampler.begin()
     for i in range(n_prof):
         flush.fill_(i & 0xFF)
         cur = x
