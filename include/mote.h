@@ -267,8 +267,9 @@ mote_status_t mote_moe_forward(const mote_layer_t* L, const void* x_bf16,
  * token on its own, so the result is bit-identical to the one-piece call): the second half's input
  * copy runs beside the first half's layer and the first half's output copy beside the second
  * half's layer, on two copy streams that the library creates on the calling thread's first such
- * call on a device and keeps.  The copies start after the work already queued on `stream`; when
- * the call returns, `stream` and both copy streams are idle. */
+ * call on a device and keeps (like the library's other per-device state they do not survive a
+ * cudaDeviceReset).  The copies start after the work already queued on `stream`; when the call
+ * returns, `stream` and both copy streams are idle. */
 size_t mote_host_staging_bytes(int d, int64_t T_max);
 mote_status_t mote_moe_forward_host(const mote_layer_t* L, const void* x_host,
                                     const void* residual_host, int64_t T, void* out_host,

@@ -235,30 +235,17 @@ __device__ __forceinline__ float glu_h(int acc_g, int acc_u, float c_g, float c_
 // for |t| > 64 where the clamp, overflow or gradual underflow could make the two differ more.
 // Flagged elements (about 0.1 %) are recomputed with glu_h.  The caller must also send rows with
 // c_g * c_u <= 1e-12 to glu_h (h' could be subnormal there).
-__device__ __forceinline__ float glu_h_fast(int acc_g, int acc_u, float c_g, float c_u, bool& redo) {
-  const float g = __fmul_rn(i2f_small(acc_g), c_g);
-  const float u = __fmul_rn(i2f_small(acc_u), c_u);
-  const float t = __fmul_rn(-g, 1.4426950408889634f);
-  float e, rc;
-  // .ftz: single instructions; with |t| <= 64 neither the operands nor the results are subnormal
-  // (a subnormal t is flushed to 0, where 2^t = 1 to well within the error budget)
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(t));
-  const float den = __fadd_rn(1.0f, e);
-  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(rc) : "f"(den));
-  const float h = __fmul_rn(u, __fmul_rn(g, rc));
-  redo = ((__float_as_uint(h) & 0xFFFFu) - 0x7FE0u) <= 0x40u || !(fabsf(t) <= 64.0f);
-  return h;
-}
-
-// glu_h_fast on raw accumulators that still carry the token's row sum (code + 1 storage): `bias` is
+// It works on raw accumulators that still carry the token's row sum (code + 1 storage): `bias` is
 // 0x4B400000 - rowsum, so that fl32(acc - rowsum) costs one integer add and one subtract per value
-// ((acc - rowsum) + 0x4B400000 == acc + bias in 32-bit arithmetic).  Same bits as glu_h_fast.
+// ((acc - rowsum) + 0x4B400000 == acc + bias in 32-bit arithmetic; see i2f_small).
 __device__ __forceinline__ float glu_h_fast_biased(uint32_t raw_g, uint32_t raw_u, uint32_t bias, float c_g, float c_u,
                                                    bool& redo) {
   const float g = __fmul_rn(__fsub_rn(__uint_as_float(raw_g + bias), kMagic), c_g);
   const float u = __fmul_rn(__fsub_rn(__uint_as_float(raw_u + bias), kMagic), c_u);
   const float t = __fmul_rn(-g, 1.4426950408889634f);
   float e, rc;
+  // .ftz: single instructions; with |t| <= 64 neither the operands nor the results are subnormal
+  // (a subnormal t is flushed to 0, where 2^t = 1 to well within the error budget)
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(t));
   const float den = __fadd_rn(1.0f, e);
   asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(rc) : "f"(den));
