@@ -250,7 +250,8 @@ __device__ __forceinline__ float glu_h_fast_biased(uint32_t raw_g, uint32_t raw_
   const float den = __fadd_rn(1.0f, e);
   asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(rc) : "f"(den));
   const float h = __fmul_rn(u, __fmul_rn(g, rc));
-  redo = ((__float_as_uint(h) & 0xFFFFu) - 0x7FE0u) <= 0x40u || !(fabsf(t) <= 64.0f);
+  // low 16 bits in [0x7FE0, 0x8020], tested in the upper half of a word: one shift-and-add, one compare
+  redo = ((__float_as_uint(h) << 16) + 0x80200000u) <= 0x00400000u || !(fabsf(t) <= 64.0f);
   return h;
 }
 
