@@ -696,8 +696,10 @@ __device__ __forceinline__ void gateup_shared_tile(const DecodeGateUpArgs& a, in
 // NTB = number of 8-token column tiles the launch is built for (1, 2, 4 or 8): ceil(T / 8) rounded up
 // kShBits = storage of the shared expert (16, 8 or 4): a kernel of its own per width, so that the
 // code expansion of the RTN widths costs the bf16 kernel no registers
+// The bf16 kernel for 9..16 tokens is held to 72 registers (it takes 80 left alone): seven CTAs per SM
+// instead of six, 8 % off the gate/up stream at T = 16.  (96 registers for 17..32 tokens: no gain.)
 template <int NTB, int kShBits>
-__global__ void __launch_bounds__(kGuWarps * 32) decode_gateup_kernel(DecodeGateUpArgs a) {
+__global__ void __launch_bounds__(kGuWarps * 32, (NTB == 2 && kShBits == 16) ? 7 : 1) decode_gateup_kernel(DecodeGateUpArgs a) {
   __shared__ ExpertList s_list;
   __shared__ float s_part[kGuWarps * NTB * 4 * 32];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;

@@ -64,6 +64,7 @@ def test_c1_full_parity(mote, path):
     (128, 320, 8, 4, 1, {}, STREAM),                      # one token, k = 4
     (896, 4864, 4, 2, 2, dict(outlier_frac=0.01), STREAM),
     (192, 320, 1, 1, 4, {}, STREAM),                      # one expert takes all four rows
+    (512, 1024, 8, 2, 13, dict(bias="zipf"), STREAM),    # 9..16 tokens: the two-column-tile kernels
 ])
 def test_small_shapes(mote, d, f, E, k, T, kw, path):
     wl = synth.custom("small", d, f, E, k, T, 2000 + d + f + T, **kw)
