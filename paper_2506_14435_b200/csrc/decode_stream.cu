@@ -73,6 +73,7 @@ struct DecodePrologueArgs {
   uint32_t* beta_h_bits;  // [T*k] zeroed here
   int32_t* rowsum_h;      // [T*k] zeroed here
   uint32_t* counter;      // zero on entry; left at zero
+  int zero_head_words;    // single-token call: words to zero from (counter - 1) on, see below; else 0
   int32_t* offsets;       // [E+1]
   int32_t* perm;          // [T*k]
   int32_t* inv;           // [T*k]
@@ -108,6 +109,11 @@ __global__ void __launch_bounds__(256) decode_prologue_kernel(DecodePrologueArgs
   // reads x too.
   pdl_wait();
   pdl_trigger();
+  // A single-token call has one prologue CTA and does not use the arrival counter, so this CTA can
+  // zero the head of the workspace (status word, counter, the down kernel's tile counters: first
+  // touched by the down kernel, which starts after this kernel has completed) instead of a memset
+  // ahead of the launch.
+  for (int i = tid; i < a.zero_head_words; i += 256) (a.counter - 1)[i] = 0u;
 
   float amax = 0.0f;
   for (int v = tid; v < n_vec; v += 256) {
@@ -949,7 +955,7 @@ mote_status_t launch_decode_stream(const DecodeStreamArgs& p, int phase, cudaStr
     pa.x = static_cast<const uint16_t*>(p.x); pa.T = T; pa.d = d; pa.E = E; pa.k = k; pa.norm_topk = p.norm_topk;
     pa.Wr = p.Wr; pa.bias = p.router_bias; pa.topk_idx = p.topk_idx; pa.topk_w = p.topk_w; pa.qx = p.qx;
     pa.beta_x = p.beta_x; pa.rowsum_x = p.rowsum_x; pa.beta_h_bits = reinterpret_cast<uint32_t*>(p.beta_h);
-    pa.rowsum_h = p.rowsum_h; pa.counter = p.counter; pa.offsets = p.offsets; pa.perm = p.perm; pa.inv = p.inv;
+    pa.rowsum_h = p.rowsum_h; pa.counter = p.counter; pa.zero_head_words = (T == 1) ? p.zero_head_words : 0; pa.offsets = p.offsets; pa.perm = p.perm; pa.inv = p.inv;
     static PerDeviceOnce prologue_attr;
     MOTE_CUDA_OK(set_max_dynamic_smem(prologue_attr, decode_prologue_kernel, 32768));
     MOTE_CUDA_OK(launch_pdl(decode_prologue_kernel, dim3(T), dim3(256), size_t(d) * 2, stream, pa));

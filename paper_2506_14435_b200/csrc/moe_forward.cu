@@ -292,9 +292,12 @@ extern "C" mote_status_t mote_moe_forward(const mote_layer_t* L, const void* x, 
   if (path == MOTE_PATH_STREAM) {
     // status word, the prologue's arrival counter, the down kernel's tile counters
     // (the kernels leave their counters at zero, so inside a stack the stack's one memset is enough)
-    if (!g_keep_status) MOTE_CUDA_OK(cudaMemsetAsync(status, 0, status_region_bytes(d), stream));
+    // (a single-token call lets its prologue kernel do it: one operation less on the stream)
+    const bool prologue_zeroes = !g_keep_status && T == 1;
+    if (!g_keep_status && !prologue_zeroes) MOTE_CUDA_OK(cudaMemsetAsync(status, 0, status_region_bytes(d), stream));
     stage_mark(0, stream);
     DecodeStreamArgs ds{};
+    ds.zero_head_words = prologue_zeroes ? int(status_region_bytes(d) / 4) : 0;
     ds.x = x; ds.T = T; ds.d = d; ds.f = f; ds.E = E; ds.k = k; ds.norm_topk = L->norm_topk;
     ds.Wr = L->Wr; ds.router_bias = L->router_bias;
     ds.gate_packed = L->gate_packed; ds.up_packed = L->up_packed; ds.down_packed = L->down_packed;

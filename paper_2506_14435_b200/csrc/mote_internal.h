@@ -127,6 +127,8 @@ struct DecodeStreamArgs {
   int8_t* qx; float* beta_x; int32_t* rowsum_x;
   void* h; int8_t* qh; float* beta_h; int32_t* rowsum_h; float* y; void* hs; float* s;
   uint32_t* counter;                       // one zeroed word
+  int zero_head_words;                     // T = 1: the prologue zeroes this many words from (counter - 1) on
+                                           // itself (status word, counter, tile counters); else 0
   uint32_t* tile_count;                    // d/16 zeroed words
   const void* residual; void* out;         // [T, d] bf16 (residual may be null, may alias out)
   int32_t* tap_gate; int32_t* tap_up; int32_t* tap_down;   // optional
