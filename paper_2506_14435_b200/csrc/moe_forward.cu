@@ -345,7 +345,10 @@ extern "C" mote_status_t mote_moe_forward(const mote_layer_t* L, const void* x, 
   }
 
   mote_status_t st;
-  if (!g_keep_status) MOTE_CUDA_OK(cudaMemsetAsync(status, 0, 4, stream));
+  // device status word: cleared by the router kernel where the tensor-core router runs (one
+  // operation less on the stream), else by a memset
+  const bool router_clears = !g_keep_status && tensor && (d % 32 == 0);
+  if (!g_keep_status && !router_clears) MOTE_CUDA_OK(cudaMemsetAsync(status, 0, 4, stream));
   stage_mark(0, stream);
   // S1 router, S2 dispatch
   // block-wise dispatch: the tensor-core router (d % 32 == 0) leaves per-block expert counts, a small
@@ -355,7 +358,7 @@ extern "C" mote_status_t mote_moe_forward(const mote_layer_t* L, const void* x, 
   auto* blk_base = reinterpret_cast<int32_t*>(base + pl.blk_base);
   const int n_blk = (int)((T + kRouteBlockTokens - 1) / kRouteBlockTokens);
   st = launch_route_topk(x, T, d, L->Wr, L->router_bias, E, k, L->norm_topk, topk_idx, topk_w, nullptr,
-                         blockwise ? blk_hist : nullptr, stream);
+                         blockwise ? blk_hist : nullptr, stream, router_clears ? status : nullptr);
   if (st) return st;
   stage_mark(1, stream);
   st = blockwise ? launch_dispatch_scan(blk_hist, n_blk, E, offsets, blk_base, tiles_routed, tiles_shared, T, stream)

@@ -39,7 +39,8 @@ __host__ __device__
 constexpr int blk_stride(int n_blk) { return (n_blk + 3) & ~3; }   // rows start on 16-byte boundaries
 mote_status_t launch_route_topk(const void* x, int64_t T, int d, const float* Wr, const float* bias,
                                 int E, int k, int norm_topk, int32_t* idx, float* w, float* logits,
-                                int32_t* blk_hist, cudaStream_t stream);
+                                int32_t* blk_hist, cudaStream_t stream, uint32_t* zero_word = nullptr);
+// zero_word (optional, tensor-core kernel only): a word the kernel's first thread sets to zero.
 
 // Stable grouping of the T*k pairs by expert: offsets[E+1], perm[P] (pair -> row), inv[P] (row -> pair).
 // Optionally also writes the 128-row tile tables of the tensor-core GEMMs ([0] = {count},

@@ -157,11 +157,14 @@ __global__ void __launch_bounds__(kRmWarps * 32, NE <= 2 ? 4 : 1) route_topk_mma
                                                                      int norm_topk, int32_t* __restrict__ idx_out,
                                                                      float* __restrict__ w_out,
                                                                      float* __restrict__ logits_out,
-                                                                     int32_t* __restrict__ blk_hist) {
+                                                                     int32_t* __restrict__ blk_hist,
+                                                                     uint32_t* __restrict__ zero_word) {
   __shared__ float s_part[kRmWarps][NE * 4][32];
   __shared__ float s_logits[16][NE * 8];
   __shared__ int s_hist[NE * 8];                      // pairs per expert among this CTA's 16 tokens
   if (threadIdx.x < NE * 8) s_hist[threadIdx.x] = 0;
+  // first kernel of a layer call on the tensor path: clears the call's device status word
+  if (zero_word && blockIdx.x == 0 && threadIdx.x == 0) *zero_word = 0u;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
   const int64_t t0 = int64_t(blockIdx.x) * 16;
   const uint16_t* xa = x + min(t0 + g, T - 1) * int64_t(d) + t * 8;       // rows past the end alias the last row
@@ -294,16 +297,16 @@ __global__ void __launch_bounds__(kRmWarps * 32, NE <= 2 ? 4 : 1) route_topk_mma
 
 mote_status_t launch_route_topk(const void* x, int64_t T, int d, const float* Wr, const float* bias, int E,
                                 int k, int norm_topk, int32_t* idx, float* w, float* logits, int32_t* blk_hist,
-                                cudaStream_t stream) {
+                                cudaStream_t stream, uint32_t* zero_word) {
   if (T == 0) return MOTE_OK;
   const uint16_t* xp = static_cast<const uint16_t*>(x);
   if (d % 32 == 0) {
     const unsigned blocks = (unsigned)((T + 15) / 16);
     const int ne = (E + 7) / 8;
-    if (ne <= 1) route_topk_mma_kernel<1><<<blocks, kRmWarps * 32, 0, stream>>>(xp, T, d, Wr, bias, E, k, norm_topk, idx, w, logits, blk_hist);
-    else if (ne <= 2) route_topk_mma_kernel<2><<<blocks, kRmWarps * 32, 0, stream>>>(xp, T, d, Wr, bias, E, k, norm_topk, idx, w, logits, blk_hist);
-    else if (ne <= 4) route_topk_mma_kernel<4><<<blocks, kRmWarps * 32, 0, stream>>>(xp, T, d, Wr, bias, E, k, norm_topk, idx, w, logits, blk_hist);
-    else route_topk_mma_kernel<8><<<blocks, kRmWarps * 32, 0, stream>>>(xp, T, d, Wr, bias, E, k, norm_topk, idx, w, logits, blk_hist);
+    if (ne <= 1) route_topk_mma_kernel<1><<<blocks, kRmWarps * 32, 0, stream>>>(xp, T, d, Wr, bias, E, k, norm_topk, idx, w, logits, blk_hist, zero_word);
+    else if (ne <= 2) route_topk_mma_kernel<2><<<blocks, kRmWarps * 32, 0, stream>>>(xp, T, d, Wr, bias, E, k, norm_topk, idx, w, logits, blk_hist, zero_word);
+    else if (ne <= 4) route_topk_mma_kernel<4><<<blocks, kRmWarps * 32, 0, stream>>>(xp, T, d, Wr, bias, E, k, norm_topk, idx, w, logits, blk_hist, zero_word);
+    else route_topk_mma_kernel<8><<<blocks, kRmWarps * 32, 0, stream>>>(xp, T, d, Wr, bias, E, k, norm_topk, idx, w, logits, blk_hist, zero_word);
   } else {
     const int per_cta = kRouteWarps * kRouteTok;
     const unsigned blocks = (unsigned)((T + per_cta - 1) / per_cta);
