@@ -704,8 +704,11 @@ __device__ __forceinline__ void gateup_shared_tile(const DecodeGateUpArgs& a, in
 // code expansion of the RTN widths costs the bf16 kernel no registers
 // The bf16 kernel for 9..16 tokens is held to 72 registers (it takes 80 left alone): seven CTAs per SM
 // instead of six, 8 % off the gate/up stream at T = 16.  (96 registers for 17..32 tokens: no gain.)
+// The other instantiations must stay without a minimum (0): a minimum of one CTA is not the same
+// to the compiler as none (it then plans for all 512 registers a thread could have, and the
+// streams of 1..8 and 17..32 tokens came out 9-50 % slower).
 template <int NTB, int kShBits>
-__global__ void __launch_bounds__(kGuWarps * 32, (NTB == 2 && kShBits == 16) ? 7 : 1) decode_gateup_kernel(DecodeGateUpArgs a) {
+__global__ void __launch_bounds__(kGuWarps * 32, (NTB == 2 && kShBits == 16) ? 7 : 0) decode_gateup_kernel(DecodeGateUpArgs a) {
   __shared__ ExpertList s_list;
   __shared__ float s_part[kGuWarps * NTB * 4 * 32];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;

@@ -18,7 +18,7 @@
 namespace mote {
 
 template <int kUnits, bool kScatter>
-__global__ void __launch_bounds__(256, kUnits <= 2 ? 4 : 1) quant_act_kernel(QuantActArgs a) {
+__global__ void __launch_bounds__(256, kUnits <= 2 ? 4 : 0) quant_act_kernel(QuantActArgs a) {
   __shared__ float s_max[8];
   __shared__ int s_sum[8];
   const int G = a.group;                          // threads per row

@@ -151,7 +151,7 @@ __device__ __forceinline__ uint32_t hi16_pair(float a, float b) {
 constexpr int kRmWarps = 8;
 
 template <int NE>   // 8-expert column tiles: ceil(E / 8) rounded up to 1, 2, 4 or 8
-__global__ void __launch_bounds__(kRmWarps * 32, NE <= 2 ? 4 : 1) route_topk_mma_kernel(const uint16_t* __restrict__ x, int64_t T, int d,
+__global__ void __launch_bounds__(kRmWarps * 32, NE <= 2 ? 4 : 0) route_topk_mma_kernel(const uint16_t* __restrict__ x, int64_t T, int d,
                                                                      const float* __restrict__ Wr,
                                                                      const float* __restrict__ bias, int E, int k,
                                                                      int norm_topk, int32_t* __restrict__ idx_out,
